@@ -1,0 +1,187 @@
+/*
+ * sp24 -- 2:4 fine-grained structured-sparse matrix multiply for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the library built from paper_2104_08378_b200/csrc.  The operations are the ones
+ * "Accelerating Sparse Deep Neural Networks" (arXiv 2104.08378) defines:
+ *
+ *   - the 2:4 pattern: in every aligned group of four consecutive values along a row at
+ *     least two are zero (Section 3, Section 3.1);
+ *   - magnitude pruning: the two smallest-magnitude values of each group of four are removed
+ *     (Section 4.1, step 2 of the workflow, Figure 5);
+ *   - the compressed format: an R x C matrix is stored as R x C/2 kept values plus 2 bits of
+ *     position metadata per kept value; a group with more than two zeros still stores two
+ *     values (Section 3.1, Figure 1);
+ *   - the sparse GEMM: sparse(M x K, stored M x K/2 + metadata) times dense(K x N) gives
+ *     dense(M x N); B and C are dense (Section 3.2, Figure 2);
+ *   - operand types FP16, BF16 (FP32 accumulate) and INT8 (INT32 accumulate) (Section 3.2,
+ *     Table 1); dimensions are multiples of 16 for 16-bit and 32 for 8-bit types (Section 3.2).
+ *
+ * Conventions that hold for every entry point unless its comment says otherwise:
+ *   - Every data pointer is a DEVICE pointer owned by the caller.  The library allocates no
+ *     device memory and frees none.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *     enqueue work; they do not synchronise.
+ *   - Argument errors are detected on the host, returned at once, and launch nothing.
+ *   - Matrices are addressed as  element(i, j) = base[i * ld + j]  for ROW_MAJOR and
+ *     base[j * ld + i] for COL_MAJOR; `ld` is in ELEMENTS.
+ *   - A (the sparse operand) is always row-major with K contiguous, because the groups of
+ *     four run along a row (Figure 1).
+ *   - The device must be compute capability 10.0 (B200); anything else gives SP24_ERR_ARCH.
+ *     There is no CPU fallback.
+ */
+#ifndef SP24_H_
+#define SP24_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SP24_OK = 0,
+  SP24_ERR_NULL = 1,        /* a required pointer is NULL                                  */
+  SP24_ERR_DTYPE = 2,       /* dtype (or dtype combination) not supported by this call     */
+  SP24_ERR_SHAPE = 3,       /* a dimension is negative or breaks the multiple-of rule      */
+  SP24_ERR_STRIDE = 4,      /* a leading dimension is too small or not 16-byte granular    */
+  SP24_ERR_ALIGN = 5,       /* a base pointer is not 16-byte aligned                       */
+  SP24_ERR_UNSUPPORTED = 6, /* valid request outside what is built (e.g. int8 alpha != 1)  */
+  SP24_ERR_WORKSPACE = 7,   /* workspace missing or smaller than sp24_gemm_workspace_bytes */
+  SP24_ERR_CUDA = 8,        /* a CUDA runtime / driver call failed                         */
+  SP24_ERR_TIMEOUT = 9,     /* a bounded device-side wait expired (see sp24_gemm_status)   */
+  SP24_ERR_ARCH = 10        /* current device is not sm_100                                */
+} sp24_status;
+
+typedef enum { SP24_F16 = 0, SP24_BF16 = 1, SP24_I8 = 2, SP24_F32 = 3, SP24_I32 = 4 } sp24_dtype;
+
+/* Metadata layouts.
+ * CANONICAL: row i occupies K/8 bytes starting at meta + i*K/8; group g of the row (columns
+ *   4g..4g+3) owns bits 4g..4g+3 of that row's little-endian bit string; the nibble is
+ *   p0 | (p1 << 2) with p0 < p1 the 0-based positions of the two kept values (Section 3.1:
+ *   the example row with indices [[0,3],[1,2]] gives nibbles 0xC, 0x9, first byte 0x9C).
+ * TCGEN05: the same nibbles permuted into the order the sm_100a sparse tensor-core
+ *   instruction reads them from tensor memory, in 2048-byte blocks of 128 rows x 128 columns
+ *   of A, rows padded to a multiple of 128 and K to a multiple of 256; padding nibbles are 0x4.
+ *   This is the layout sp24_gemm consumes. */
+typedef enum { SP24_META_CANONICAL = 0, SP24_META_TCGEN05 = 1 } sp24_meta_layout;
+
+/* Which index of a matrix is contiguous in memory. */
+typedef enum { SP24_ROW_MAJOR = 0, SP24_COL_MAJOR = 1 } sp24_order;
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* sp24_status_string(sp24_status s);
+
+/* Bytes of the kept-value array of an M x K matrix: M * (K/2) * sizeof(t)  (Figure 1:
+ * R x C becomes R x C/2).  Returns 0 for an unsupported dtype or K % 4 != 0. */
+size_t sp24_values_bytes(sp24_dtype t, int64_t M, int64_t K);
+
+/* Bytes of the metadata of an M x K matrix.  CANONICAL: M*K/8 (2 bits per kept value,
+ * Section 3.1, i.e. 12.5 % / 25 % of the kept values for 16-bit / 8-bit types).
+ * TCGEN05: ceil(M/128) * ceil(K/256) * 4096.  Returns 0 for bad arguments. */
+size_t sp24_meta_bytes(sp24_dtype t, int64_t M, int64_t K, sp24_meta_layout l);
+
+/* Magnitude pruning to 2:4 (Section 4.1 step 2; pattern of Section 3).
+ * For every row i < M and every aligned group of four columns 4g..4g+3 < K the two values of
+ * largest magnitude are copied bit-for-bit to y, the other two positions receive +0.  Equal
+ * magnitudes: the lower column index is kept.  Magnitude is |x| for I8 (so -128 ranks as
+ * 128) and the bit pattern without its sign bit for F16/BF16 (denormals are not flushed).
+ *   t: SP24_F16, SP24_BF16 or SP24_I8.      M >= 0, K >= 0, K % 4 == 0.
+ *   x: device, M x K row-major, leading dimension ldx >= K (elements).
+ *   y: device, same shape, leading dimension ldy >= K; may be the same buffer as x.
+ * Fastest when x, y are 16-byte aligned and ldx*sizeof(t), ldy*sizeof(t), K*sizeof(t) are
+ * multiples of 16; other cases take a scalar path with the same result. */
+sp24_status sp24_prune(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx,
+                       void* y, int64_t ldy, void* stream);
+
+/* Compression to kept values + metadata (Section 3.1, Figure 1).
+ * Applies the selection rule of sp24_prune to x itself, so compress(x) == compress(prune(x))
+ * and the call doubles as the fused prune+compress pass.  For group g of row i with kept
+ * positions p0 < p1:  vals[i*ldv + 2g] = x[i, 4g+p0],  vals[i*ldv + 2g+1] = x[i, 4g+p1],
+ * metadata nibble p0 | (p1<<2) stored as `l` says.  A group with fewer than two non-zeros is
+ * completed with its lowest-index zeros (an all-zero group stores positions 0,1).
+ *   vals: device, M x K/2 row-major, ldv >= K/2 (elements).
+ *   meta: device, sp24_meta_bytes(t, M, K, l) bytes; for TCGEN05 the padding is written too.
+ *   dropped_nonzeros: device counter or NULL.  If given, the number of non-kept positions
+ *     holding a non-zero magnitude is ADDED to it (0 added iff x already was 2:4).
+ * Requires K % 4 == 0 (K % 16 == 0 for the vectorised path). */
+sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx,
+                          void* vals, int64_t ldv, void* meta, sp24_meta_layout l,
+                          unsigned long long* dropped_nonzeros, void* stream);
+
+/* Inverse of sp24_compress (the metadata "decodes the compressed format", Section 3.1):
+ * y is M x K row-major (ldy >= K) with y[i, 4g+p_t] = vals[i, 2g+t] and +0 elsewhere. */
+sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals, int64_t ldv,
+                            const void* meta, sp24_meta_layout l, void* y, int64_t ldy,
+                            void* stream);
+
+/* Problem description of D = alpha * op(A) * B + beta * C  (Section 3.2, Figure 2).
+ *   ab_type: SP24_F16 or SP24_BF16 (FP32 accumulate) or SP24_I8 (INT32 accumulate) -- the
+ *            operand/accumulator pairs of Table 1.
+ *   cd_type: type of C and D.  F16/BF16 operands: SP24_F16, SP24_BF16 (ab_type's own) or
+ *            SP24_F32.  I8 operands: SP24_I32.
+ *   M, N, K: K is the LOGICAL (uncompressed) reduction length.  M, N, K must be multiples of
+ *            16 (16-bit types) or 32 (I8) (Section 3.2); zero-sized problems return SP24_OK.
+ *   lda:     leading dimension of the A-side value array: of vals (M x K/2) when
+ *            a_is_dense == 0, of the dense M x K matrix when a_is_dense == 1.
+ *   order_b: SP24_COL_MAJOR = K contiguous (B stored as N rows of K values: the
+ *            [tokens, hidden] activation layout), the only order built so far.
+ *   order_c / order_d: SP24_ROW_MAJOR (N contiguous).
+ *   a_is_dense: 0 = 2:4 compressed A with TCGEN05 metadata (the sparse tensor-core path);
+ *            1 = the dense variant on the same pipeline (`A` is M x K dense, `meta` unused).
+ * All leading dimensions are in elements and, in bytes, multiples of 16. */
+typedef struct {
+  sp24_dtype ab_type, cd_type;
+  int64_t M, N, K;
+  int64_t lda, ldb, ldc, ldd;
+  sp24_order order_b, order_c, order_d;
+  int a_is_dense;
+} sp24_gemm_desc;
+
+/* Bytes of device workspace sp24_gemm needs for this problem (currently a fixed 256 bytes:
+ * the device-side status record).  The workspace must be 16-byte aligned. */
+size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d);
+
+/* The 2:4 sparse GEMM on the sparse tensor cores (Section 3.2, Figure 2):
+ *   D[i,j] = alpha * sum_g sum_{t=0,1} vals[i,2g+t] * B[4g + p_t(i,g), j] + beta * C[i,j].
+ *   alpha, beta: HOST pointers.  float for F16/BF16 operands; int32_t for I8, where only
+ *                alpha == 1 and beta in {0, 1} are built (else SP24_ERR_UNSUPPORTED).
+ *   A:    device; vals (M x K/2) or dense A (M x K), row-major, 16-byte aligned.
+ *   meta: device; TCGEN05-layout metadata of A (ignored when a_is_dense).
+ *   B, C, D: device, 16-byte aligned.  C may be NULL iff beta == 0.  C may alias D.
+ *   workspace: device, >= sp24_gemm_workspace_bytes(d).  The kernel writes a status record
+ *              there; read it back with sp24_gemm_status after synchronising.
+ * Accumulation is FP32 (INT32) in hardware order; the result is rounded to cd_type once,
+ * round-to-nearest-even. */
+sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A,
+                      const void* meta, const void* B, const void* beta, const void* C,
+                      void* D, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Copies the status record of the last sp24_gemm that used `workspace` back to the host
+ * (synchronises `stream`) and returns SP24_OK, or SP24_ERR_TIMEOUT if a bounded wait inside
+ * the kernel expired (the kernel then returned early and D is incomplete). */
+sp24_status sp24_gemm_status(const void* workspace, void* stream);
+
+/* Lowering of a 3x3, stride-1, pad-1 NHWC convolution input to the GEMM's B operand
+ * (Section 4.2: a convolution's reduction dimension is C*R*S).  Output is K-contiguous:
+ *   out[((n*H + h)*W + w) * ldo + (r*3 + s)*C + c] = in[n, h+r-1, w+s-1, c]  (0 outside).
+ *   t: SP24_F16, SP24_BF16 or SP24_I8.  C*sizeof(t) must be a multiple of 16; ldo >= 9*C. */
+sp24_status sp24_im2col_nhwc_3x3(sp24_dtype t, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                                 const void* in, void* out, int64_t ldo, void* stream);
+
+/* End-to-end convenience for callers whose data lives in HOST memory (pinned for speed):
+ * copies dense A (M x K, row-major, packed), B (N rows of K, packed) and, if beta != 0, C
+ * (M x N packed) to the device buffers the caller provides, runs sp24_compress (TCGEN05
+ * layout) and sp24_gemm, and copies D (M x N packed) back.  All h_* are host pointers, all
+ * d_* device pointers sized for the packed matrices (d_vals, d_meta as the size helpers
+ * say).  Work is enqueued on `stream`; the caller synchronises. */
+sp24_status sp24_pipeline_host(const sp24_gemm_desc* d, const void* alpha, const void* h_A,
+                               const void* h_B, const void* beta, const void* h_C, void* h_D,
+                               void* d_A, void* d_vals, void* d_meta, void* d_B, void* d_C,
+                               void* d_D, void* workspace, size_t workspace_bytes,
+                               void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SP24_H_ */

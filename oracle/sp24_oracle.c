@@ -1,0 +1,376 @@
+/*
+ * CPU oracle for the 2:4 structured-sparse path of "Accelerating Sparse Deep Neural
+ * Networks" (arXiv 2104.08378).
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a plain, slow, scalar restatement of
+ * what the path computes, written from the paper, and shares no code with the CUDA library.
+ * Only the tests, the smoke check and the bench's CPU-baseline / reference legs may call it.
+ *
+ * Every function walks the definition directly: one loop per index, no blocking, no fusion.
+ * Floating-point GEMMs read the fp16 / bf16 inputs exactly into double and accumulate in
+ * double; the int8 GEMM accumulates in int64.  The only concession to run time is an OpenMP
+ * "parallel for" over output rows (rows are independent in every operation here).
+ *
+ * dtype codes: 0 = fp16, 1 = bf16, 2 = int8.  Matrices are row-major with a leading
+ * dimension in elements unless stated.
+ *
+ * Pins (tests/test_oracle_*.py): the pattern invariant and idempotence, brute force over all
+ * C(4,2) keep-patterns, the metadata example of Section 3.1, the storage arithmetic of
+ * Section 3.1, decompress(compress(x)) == prune(x), sparse GEMM == library dense matmul on
+ * the pruned matrix, closed forms (identity B, all-ones), a direct 7-loop convolution for
+ * im2col, and hand-computed positions for the tensor-core metadata permutation.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ------------------------------------------------------------------------------------- */
+/* element helpers                                                                       */
+/* ------------------------------------------------------------------------------------- */
+
+static int elem_size(int dtype) { return dtype == 2 ? 1 : 2; }
+
+/* IEEE binary16 bit pattern -> double, exactly. */
+static double half_bits_to_double(uint16_t h) {
+  int sign = (h >> 15) & 1;
+  int exponent = (h >> 10) & 0x1F;
+  int mantissa = h & 0x3FF;
+  double v;
+  if (exponent == 0) {
+    v = ldexp((double)mantissa, -24); /* zero and subnormals: mantissa * 2^-24 */
+  } else if (exponent == 31) {
+    v = mantissa ? NAN : INFINITY;
+  } else {
+    v = ldexp((double)(mantissa + 1024), exponent - 25); /* (1 + m/1024) * 2^(e-15) */
+  }
+  return sign ? -v : v;
+}
+
+/* bfloat16 bit pattern -> double, exactly: bf16 is the upper half of an IEEE binary32. */
+static double bf16_bits_to_double(uint16_t b) {
+  uint32_t w = ((uint32_t)b) << 16;
+  float f;
+  memcpy(&f, &w, sizeof f);
+  return (double)f;
+}
+
+static double load_as_double(int dtype, const void* base, int64_t index) {
+  if (dtype == 0) return half_bits_to_double(((const uint16_t*)base)[index]);
+  if (dtype == 1) return bf16_bits_to_double(((const uint16_t*)base)[index]);
+  return (double)((const int8_t*)base)[index];
+}
+
+/* Magnitude key used by the pruning criterion (Section 4.1, step 2: "magnitude").
+ * 16-bit floats: the bit pattern without the sign bit, which orders finite values by |x|
+ * (zero of either sign -> 0, subnormals keep their rank).  int8: |x| as an int, -128 -> 128. */
+static int magnitude_key(int dtype, const void* base, int64_t index) {
+  if (dtype == 2) {
+    int v = ((const int8_t*)base)[index];
+    return v < 0 ? -v : v;
+  }
+  return ((const uint16_t*)base)[index] & 0x7FFF;
+}
+
+/* The two kept positions of one group of four (Section 4.1 step 2: the two smallest are
+ * removed; ties keep the lower index).  Rank each position by how many others beat it: j
+ * beats p if its key is larger, or equal with a smaller index.  Positions with rank 0 and 1
+ * are kept; they are returned in ascending order p0 < p1 (Section 3.1 lists indices in
+ * ascending order inside a group). */
+static void select_two(const int key[4], int* p0, int* p1) {
+  int kept[2];
+  int n = 0;
+  for (int p = 0; p < 4; ++p) {
+    int beaten_by = 0;
+    for (int j = 0; j < 4; ++j) {
+      if (j == p) continue;
+      if (key[j] > key[p] || (key[j] == key[p] && j < p)) ++beaten_by;
+    }
+    if (beaten_by < 2) kept[n++] = p;
+  }
+  *p0 = kept[0];
+  *p1 = kept[1];
+}
+
+static void copy_elem(int dtype, void* dst, int64_t di, const void* src, int64_t si) {
+  if (dtype == 2) ((int8_t*)dst)[di] = ((const int8_t*)src)[si];
+  else ((uint16_t*)dst)[di] = ((const uint16_t*)src)[si];
+}
+
+static void zero_elem(int dtype, void* dst, int64_t di) {
+  if (dtype == 2) ((int8_t*)dst)[di] = 0;
+  else ((uint16_t*)dst)[di] = 0; /* +0 */
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------------------------- */
+/* prune  (Section 3 pattern; Section 4.1 step 2)                                        */
+/* ------------------------------------------------------------------------------------- */
+void oracle_prune(int dtype, int64_t M, int64_t K, const void* x, int64_t ldx, void* y,
+                  int64_t ldy) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < M; ++i) {
+    for (int64_t g = 0; g < K / 4; ++g) {
+      int key[4], p0, p1;
+      for (int p = 0; p < 4; ++p) key[p] = magnitude_key(dtype, x, i * ldx + 4 * g + p);
+      select_two(key, &p0, &p1);
+      for (int p = 0; p < 4; ++p) {
+        if (p == p0 || p == p1) copy_elem(dtype, y, i * ldy + 4 * g + p, x, i * ldx + 4 * g + p);
+        else zero_elem(dtype, y, i * ldy + 4 * g + p);
+      }
+    }
+  }
+}
+
+/* ------------------------------------------------------------------------------------- */
+/* compress  (Section 3.1, Figure 1)                                                      */
+/* vals is M x K/2; meta is the canonical layout: K/8 bytes per row, group g in bits       */
+/* 4g..4g+3 of the row's little-endian bit string, nibble = p0 | p1 << 2.                  */
+/* Returns the number of dropped positions whose magnitude was non-zero.                   */
+/* ------------------------------------------------------------------------------------- */
+int64_t oracle_compress(int dtype, int64_t M, int64_t K, const void* x, int64_t ldx, void* vals,
+                        int64_t ldv, uint8_t* meta) {
+  int64_t dropped = 0;
+  memset(meta, 0, (size_t)(M * (K / 8)));
+#pragma omp parallel for schedule(static) reduction(+ : dropped)
+  for (int64_t i = 0; i < M; ++i) {
+    for (int64_t g = 0; g < K / 4; ++g) {
+      int key[4], p0, p1;
+      for (int p = 0; p < 4; ++p) key[p] = magnitude_key(dtype, x, i * ldx + 4 * g + p);
+      select_two(key, &p0, &p1);
+      copy_elem(dtype, vals, i * ldv + 2 * g, x, i * ldx + 4 * g + p0);
+      copy_elem(dtype, vals, i * ldv + 2 * g + 1, x, i * ldx + 4 * g + p1);
+      uint8_t nibble = (uint8_t)(p0 | (p1 << 2));
+      meta[i * (K / 8) + g / 2] |= (uint8_t)(nibble << (4 * (g % 2)));
+      for (int p = 0; p < 4; ++p)
+        if (p != p0 && p != p1 && key[p] != 0) ++dropped;
+    }
+  }
+  return dropped;
+}
+
+static void nibble_positions(const uint8_t* meta, int64_t K, int64_t i, int64_t g, int* p0,
+                             int* p1) {
+  uint8_t byte = meta[i * (K / 8) + g / 2];
+  int nibble = (byte >> (4 * (g % 2))) & 0xF;
+  *p0 = nibble & 3;
+  *p1 = (nibble >> 2) & 3;
+}
+
+/* ------------------------------------------------------------------------------------- */
+/* decompress: the metadata decodes the compressed format (Section 3.1)                   */
+/* ------------------------------------------------------------------------------------- */
+void oracle_decompress(int dtype, int64_t M, int64_t K, const void* vals, int64_t ldv,
+                       const uint8_t* meta, void* y, int64_t ldy) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < M; ++i) {
+    for (int64_t k = 0; k < K; ++k) zero_elem(dtype, y, i * ldy + k);
+    for (int64_t g = 0; g < K / 4; ++g) {
+      int p0, p1;
+      nibble_positions(meta, K, i, g, &p0, &p1);
+      copy_elem(dtype, y, i * ldy + 4 * g + p0, vals, i * ldv + 2 * g);
+      copy_elem(dtype, y, i * ldy + 4 * g + p1, vals, i * ldv + 2 * g + 1);
+    }
+  }
+}
+
+/* ------------------------------------------------------------------------------------- */
+/* Tensor-core operand order of the metadata.                                             */
+/* The nibbles of the canonical layout, permuted into 2048-byte blocks that each cover     */
+/* 128 rows x 128 columns of A.  Rows are padded to a multiple of 128 and K to a multiple  */
+/* of 256; padding nibbles are 0x4 (positions 0,1).  Block (mb, kb) starts at byte         */
+/* (mb * KB + kb) * 2048 with KB = 2 * ceil(K / 256).  Inside a block, for local row r,    */
+/* local group q (0..31):                                                                  */
+/*   int8:  bit = 128*r + 4*q                                                              */
+/*   16-bit types: rows are paired (r, r+8) inside each 16-row band and the two 16-column  */
+/*          halves of every 32-column slice are split across lanes:                        */
+/*          bit = 128*(r%8) + 16*((r/8)%2) + 2048*(r/16)                                   */
+/*              + 1024*((q/4)%2) + 32*(q/8) + 4*(q%4)                                      */
+/* direction 0: canonical -> operand order, 1: operand order -> canonical.                 */
+/* ------------------------------------------------------------------------------------- */
+static int64_t operand_bit_in_block(int dtype, int r, int q) {
+  if (dtype == 2) return 128 * (int64_t)r + 4 * q;
+  return 128 * (r % 8) + 16 * ((r / 8) % 2) + 2048 * (r / 16) + 1024 * ((q / 4) % 2) +
+         32 * (q / 8) + 4 * (q % 4);
+}
+
+int64_t oracle_meta_operand_bytes(int64_t M, int64_t K) {
+  int64_t MB = (M + 127) / 128, KB = 2 * ((K + 255) / 256);
+  return MB * KB * 2048;
+}
+
+void oracle_meta_permute(int dtype, int64_t M, int64_t K, const uint8_t* src, uint8_t* dst,
+                         int direction) {
+  int64_t MB = (M + 127) / 128, KB = 2 * ((K + 255) / 256);
+  if (direction == 0) memset(dst, 0x44, (size_t)(MB * KB * 2048));
+  else memset(dst, 0, (size_t)(M * (K / 8)));
+  for (int64_t i = 0; i < M; ++i) {
+    for (int64_t g = 0; g < K / 4; ++g) {
+      int64_t mb = i / 128, kb = g / 32;
+      int r = (int)(i % 128), q = (int)(g % 32);
+      int64_t bit = ((mb * KB + kb) * 2048) * 8 + operand_bit_in_block(dtype, r, q);
+      int64_t cbyte = i * (K / 8) + g / 2;
+      int cshift = 4 * (int)(g % 2);
+      int64_t obyte = bit / 8;
+      int oshift = (int)(bit % 8);
+      if (direction == 0) {
+        int nibble = (src[cbyte] >> cshift) & 0xF;
+        dst[obyte] = (uint8_t)((dst[obyte] & ~(0xF << oshift)) | (nibble << oshift));
+      } else {
+        int nibble = (src[obyte] >> oshift) & 0xF;
+        dst[cbyte] |= (uint8_t)(nibble << cshift);
+      }
+    }
+  }
+}
+
+/* ------------------------------------------------------------------------------------- */
+/* GEMM  (Section 3.2, Figure 2)                                                           */
+/* D[i,j] = alpha * sum_g sum_t vals[i,2g+t] * B[4g+p_t(i,g), j] + beta * C[i,j]           */
+/* on the output window rows [i0,i1) x columns [j0,j1); out is (i1-i0) x (j1-j0) packed.   */
+/* B element (k, j) is B[k + j*ldb] when b_k_contiguous, else B[k*ldb + j].                */
+/* C element (i, j) is C[i*ldc + j]; c_dtype codes: 0 fp16, 1 bf16, 3 fp32, 4 int32.       */
+/* Floating point: out_f64 receives the un-rounded double result.                          */
+/* int8: exact int64 accumulation, out_i32 receives the value cast to int32.               */
+/* ------------------------------------------------------------------------------------- */
+static double load_c(int c_dtype, const void* C, int64_t index) {
+  if (c_dtype == 0) return half_bits_to_double(((const uint16_t*)C)[index]);
+  if (c_dtype == 1) return bf16_bits_to_double(((const uint16_t*)C)[index]);
+  if (c_dtype == 3) return (double)((const float*)C)[index];
+  return (double)((const int32_t*)C)[index];
+}
+
+void oracle_gemm_sparse(int dtype, int64_t M, int64_t N, int64_t K, const void* vals,
+                        int64_t ldv, const uint8_t* meta, const void* B, int64_t ldb,
+                        int b_k_contiguous, double alpha, double beta, int c_dtype,
+                        const void* C, int64_t ldc, int64_t i0, int64_t i1, int64_t j0,
+                        int64_t j1, double* out_f64, int32_t* out_i32) {
+  (void)M;
+  (void)N;
+  int64_t width = j1 - j0;
+#pragma omp parallel for schedule(dynamic, 4)
+  for (int64_t i = i0; i < i1; ++i) {
+    for (int64_t j = j0; j < j1; ++j) {
+      double acc = 0.0;
+      int64_t iacc = 0;
+      for (int64_t g = 0; g < K / 4; ++g) {
+        int p[2];
+        nibble_positions(meta, K, i, g, &p[0], &p[1]);
+        for (int t = 0; t < 2; ++t) {
+          int64_t k = 4 * g + p[t];
+          int64_t bidx = b_k_contiguous ? k + j * ldb : k * ldb + j;
+          if (dtype == 2) {
+            iacc += (int64_t)((const int8_t*)vals)[i * ldv + 2 * g + t] *
+                    (int64_t)((const int8_t*)B)[bidx];
+          } else {
+            acc += load_as_double(dtype, vals, i * ldv + 2 * g + t) * load_as_double(dtype, B, bidx);
+          }
+        }
+      }
+      int64_t o = (i - i0) * width + (j - j0);
+      if (dtype == 2) {
+        int64_t r = (int64_t)alpha * iacc;
+        if (beta != 0.0 && C) r += (int64_t)beta * (int64_t)((const int32_t*)C)[i * ldc + j];
+        out_i32[o] = (int32_t)r;
+      } else {
+        double r = alpha * acc;
+        if (beta != 0.0 && C) r += beta * load_c(c_dtype, C, i * ldc + j);
+        out_f64[o] = r;
+      }
+    }
+  }
+}
+
+/* The textbook dense product on a dense A (used on prune(x) and on decompress(...)):
+ * D[i,j] = alpha * sum_k A[i,k] * B[k,j] + beta * C[i,j], k ascending. */
+void oracle_gemm_dense(int dtype, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                       const void* B, int64_t ldb, int b_k_contiguous, double alpha, double beta,
+                       int c_dtype, const void* C, int64_t ldc, int64_t i0, int64_t i1,
+                       int64_t j0, int64_t j1, double* out_f64, int32_t* out_i32) {
+  (void)M;
+  (void)N;
+  int64_t width = j1 - j0;
+#pragma omp parallel for schedule(dynamic, 4)
+  for (int64_t i = i0; i < i1; ++i) {
+    for (int64_t j = j0; j < j1; ++j) {
+      double acc = 0.0;
+      int64_t iacc = 0;
+      for (int64_t k = 0; k < K; ++k) {
+        int64_t bidx = b_k_contiguous ? k + j * ldb : k * ldb + j;
+        if (dtype == 2) {
+          iacc += (int64_t)((const int8_t*)A)[i * lda + k] * (int64_t)((const int8_t*)B)[bidx];
+        } else {
+          acc += load_as_double(dtype, A, i * lda + k) * load_as_double(dtype, B, bidx);
+        }
+      }
+      int64_t o = (i - i0) * width + (j - j0);
+      if (dtype == 2) {
+        int64_t r = (int64_t)alpha * iacc;
+        if (beta != 0.0 && C) r += (int64_t)beta * (int64_t)((const int32_t*)C)[i * ldc + j];
+        out_i32[o] = (int32_t)r;
+      } else {
+        double r = alpha * acc;
+        if (beta != 0.0 && C) r += beta * load_c(c_dtype, C, i * ldc + j);
+        out_f64[o] = r;
+      }
+    }
+  }
+}
+
+/* sum_k |A[i,k]| * |B[k,j]| over the kept values, in double: the scale of the per-element
+ * error bound for the floating-point GEMM. */
+void oracle_gemm_abs(int dtype, int64_t K, const void* vals, int64_t ldv, const uint8_t* meta,
+                     const void* B, int64_t ldb, int b_k_contiguous, int64_t i0, int64_t i1,
+                     int64_t j0, int64_t j1, double* out_f64) {
+  int64_t width = j1 - j0;
+#pragma omp parallel for schedule(dynamic, 4)
+  for (int64_t i = i0; i < i1; ++i) {
+    for (int64_t j = j0; j < j1; ++j) {
+      double acc = 0.0;
+      for (int64_t g = 0; g < K / 4; ++g) {
+        int p[2];
+        nibble_positions(meta, K, i, g, &p[0], &p[1]);
+        for (int t = 0; t < 2; ++t) {
+          int64_t k = 4 * g + p[t];
+          int64_t bidx = b_k_contiguous ? k + j * ldb : k * ldb + j;
+          acc += fabs(load_as_double(dtype, vals, i * ldv + 2 * g + t)) *
+                 fabs(load_as_double(dtype, B, bidx));
+        }
+      }
+      out_f64[(i - i0) * width + (j - j0)] = acc;
+    }
+  }
+}
+
+/* ------------------------------------------------------------------------------------- */
+/* im2col for a 3x3, stride 1, pad 1 convolution on NHWC input (Section 4.2: the           */
+/* reduction dimension of a convolution is C*R*S).  K index = (r*3 + s)*C + c, output      */
+/* column = (n*H + h)*W + w, stored K-contiguous with leading dimension ldo.               */
+/* ------------------------------------------------------------------------------------- */
+void oracle_im2col_nhwc_3x3(int dtype, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                            const void* in, void* out, int64_t ldo) {
+#pragma omp parallel for schedule(static)
+  for (int64_t n = 0; n < Nb; ++n)
+    for (int64_t h = 0; h < H; ++h)
+      for (int64_t w = 0; w < W; ++w)
+        for (int r = 0; r < 3; ++r)
+          for (int s = 0; s < 3; ++s)
+            for (int64_t c = 0; c < C; ++c) {
+              int64_t hh = h + r - 1, ww = w + s - 1;
+              int64_t o = ((n * H + h) * W + w) * ldo + (r * 3 + s) * C + c;
+              if (hh < 0 || hh >= H || ww < 0 || ww >= W) zero_elem(dtype, out, o);
+              else copy_elem(dtype, out, o, in, ((n * H + hh) * W + ww) * C + c);
+            }
+}
+
+int oracle_elem_size(int dtype) { return elem_size(dtype); }

@@ -1,0 +1,70 @@
+/*
+ * Stateless counter-based generator for the synthetic benchmark inputs (host side, plain C).
+ * Holds none of the method's arithmetic.  Element `index` of tensor `tensor_id` under `seed`
+ * depends on nothing else, so any slice of a matrix can be regenerated on its own.
+ *
+ * kinds: 0 = N(0, p0) by Box-Muller, 1 = U(p0, p1), 2 = integers uniform in [-127, 127],
+ *        3 = max(N(0, p0), 0).
+ * dtype: 0 = fp16 bits, 1 = bf16 bits (both round-to-nearest-even), 2 = int8.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+static uint64_t mix64(uint64_t z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+  return z ^ (z >> 31);
+}
+
+static uint64_t stream_key(uint64_t seed, uint64_t tensor_id, uint64_t stream) {
+  return mix64(seed * 0x100000001B3ULL + tensor_id * 0x9E37ULL + stream * 0x51ED27ULL +
+               0x9E3779B97F4A7C15ULL);
+}
+
+uint64_t sp24_inputs_raw(uint64_t seed, uint64_t tensor_id, uint64_t stream, uint64_t index) {
+  return mix64(index * 0x9E3779B97F4A7C15ULL + stream_key(seed, tensor_id, stream));
+}
+
+static double unit_open(uint64_t u) { /* (0,1): 53 bits, offset by half a step */
+  return ((double)(u >> 11) + 0.5) * (1.0 / 9007199254740992.0);
+}
+
+static uint16_t float_to_bf16_rne(float f) {
+  uint32_t bits;
+  memcpy(&bits, &f, 4);
+  if ((bits & 0x7F800000u) == 0x7F800000u) return (uint16_t)(bits >> 16); /* inf / nan */
+  bits += 0x7FFFu + ((bits >> 16) & 1u);
+  return (uint16_t)(bits >> 16);
+}
+
+static uint16_t double_to_half_rne(double d) {
+  /* _Float16 conversion from double rounds once, to nearest even. */
+  _Float16 h = (_Float16)d;
+  uint16_t bits;
+  memcpy(&bits, &h, 2);
+  return bits;
+}
+
+void sp24_inputs_fill(int kind, double p0, double p1, int dtype, uint64_t seed,
+                      uint64_t tensor_id, uint64_t start, uint64_t count, void* out) {
+  const uint64_t k0 = stream_key(seed, tensor_id, 0), k1 = stream_key(seed, tensor_id, 1);
+#pragma omp parallel for schedule(static)
+  for (int64_t n = 0; n < (int64_t)count; ++n) {
+    uint64_t idx = (start + (uint64_t)n) * 0x9E3779B97F4A7C15ULL;
+    uint64_t a = mix64(idx + k0);
+    double v;
+    if (kind == 2) {
+      v = (double)((int)(a % 255u) - 127);
+    } else if (kind == 1) {
+      v = p0 + (p1 - p0) * unit_open(a);
+    } else {
+      uint64_t b = mix64(idx + k1);
+      v = p0 * sqrt(-2.0 * log(unit_open(a))) * cos(6.283185307179586476925 * unit_open(b));
+      if (kind == 3 && v < 0.0) v = 0.0;
+    }
+    if (dtype == 2) ((int8_t*)out)[n] = (int8_t)v;
+    else if (dtype == 1) ((uint16_t*)out)[n] = float_to_bf16_rne((float)v);
+    else ((uint16_t*)out)[n] = double_to_half_rne(v);
+  }
+}

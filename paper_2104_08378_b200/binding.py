@@ -1,0 +1,208 @@
+"""ctypes binding of the sp24 C ABI (include/sp24.h): argument marshalling only.
+
+Every function takes torch CUDA tensors (PyTorch is used for device memory and streams only),
+passes their device pointers and the current stream to ``libsp24.so`` and raises
+``Sp24Error`` on a non-zero status.  There is no CPU fallback: if the library is missing the
+import fails, and every call needs a CUDA device.
+
+16-bit matrices may be torch.float16 / torch.bfloat16 or raw torch.int16 / uint16 bit patterns
+(then pass ``dtype=`` explicitly); int8 matrices are torch.int8.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from .build import LIB_PATH
+
+OK = 0
+F16, BF16, I8, F32, I32 = 0, 1, 2, 3, 4
+META_CANONICAL, META_TCGEN05 = 0, 1
+ROW_MAJOR, COL_MAJOR = 0, 1
+DTYPE_CODE = {"f16": F16, "bf16": BF16, "i8": I8, "f32": F32, "i32": I32}
+TORCH_DTYPE = {"f16": torch.float16, "bf16": torch.bfloat16, "i8": torch.int8, "f32": torch.float32,
+               "i32": torch.int32}
+_FROM_TORCH = {torch.float16: "f16", torch.bfloat16: "bf16", torch.int8: "i8", torch.float32: "f32",
+               torch.int32: "i32"}
+
+EXPORTS = [
+    "sp24_status_string", "sp24_values_bytes", "sp24_meta_bytes", "sp24_prune", "sp24_compress",
+    "sp24_decompress", "sp24_gemm_workspace_bytes", "sp24_gemm", "sp24_gemm_status",
+    "sp24_im2col_nhwc_3x3", "sp24_pipeline_host",
+]
+
+
+class Sp24Error(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: sp24 status {status} ({status_string(status)})")
+
+
+class GemmDesc(ctypes.Structure):
+    _fields_ = [("ab_type", ctypes.c_int), ("cd_type", ctypes.c_int),
+                ("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("lda", ctypes.c_int64), ("ldb", ctypes.c_int64), ("ldc", ctypes.c_int64),
+                ("ldd", ctypes.c_int64),
+                ("order_b", ctypes.c_int), ("order_c", ctypes.c_int), ("order_d", ctypes.c_int),
+                ("a_is_dense", ctypes.c_int)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2104_08378_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    i64, vp, ci, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.sp24_status_string.argtypes = [ci]
+    lib.sp24_status_string.restype = ctypes.c_char_p
+    lib.sp24_values_bytes.argtypes = [ci, i64, i64]
+    lib.sp24_values_bytes.restype = sz
+    lib.sp24_meta_bytes.argtypes = [ci, i64, i64, ci]
+    lib.sp24_meta_bytes.restype = sz
+    lib.sp24_prune.argtypes = [ci, i64, i64, vp, i64, vp, i64, vp]
+    lib.sp24_compress.argtypes = [ci, i64, i64, vp, i64, vp, i64, vp, ci, vp, vp]
+    lib.sp24_decompress.argtypes = [ci, i64, i64, vp, i64, vp, ci, vp, i64, vp]
+    lib.sp24_gemm_workspace_bytes.argtypes = [ctypes.POINTER(GemmDesc)]
+    lib.sp24_gemm_workspace_bytes.restype = sz
+    lib.sp24_gemm.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sp24_gemm_status.argtypes = [vp, vp]
+    lib.sp24_im2col_nhwc_3x3.argtypes = [ci, i64, i64, i64, i64, vp, vp, i64, vp]
+    lib.sp24_pipeline_host.argtypes = [ctypes.POINTER(GemmDesc)] + [vp] * 13 + [sz, vp]
+    for name in ("sp24_prune", "sp24_compress", "sp24_decompress", "sp24_gemm", "sp24_gemm_status",
+                 "sp24_im2col_nhwc_3x3", "sp24_pipeline_host"):
+        getattr(lib, name).restype = ci
+    return lib
+
+
+lib = _load()
+
+
+def status_string(status: int) -> str:
+    return lib.sp24_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise Sp24Error(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dtype_of(t: torch.Tensor, dtype: str | None) -> str:
+    if dtype is not None:
+        return dtype
+    return _FROM_TORCH[t.dtype]
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def values_bytes(dtype: str, M: int, K: int) -> int:
+    return lib.sp24_values_bytes(DTYPE_CODE[dtype], M, K)
+
+
+def meta_bytes(dtype: str, M: int, K: int, layout: int = META_TCGEN05) -> int:
+    return lib.sp24_meta_bytes(DTYPE_CODE[dtype], M, K, layout)
+
+
+def prune(x: torch.Tensor, out: torch.Tensor | None = None, dtype: str | None = None) -> torch.Tensor:
+    """sp24_prune on a 2-D row-major tensor (row stride = leading dimension)."""
+    dt = _dtype_of(x, dtype)
+    M, K = x.shape
+    if out is None:
+        out = torch.empty((M, K), dtype=x.dtype, device=x.device)
+    assert x.stride(1) == 1 or K <= 1
+    _check(lib.sp24_prune(DTYPE_CODE[dt], M, K, _ptr(x), x.stride(0) if M > 1 else K, _ptr(out),
+                          out.stride(0) if M > 1 else K, _stream()), "sp24_prune")
+    return out
+
+
+def compress(x: torch.Tensor, layout: int = META_TCGEN05, dtype: str | None = None,
+             count_dropped: bool = False):
+    """sp24_compress: returns (vals [M, K/2], meta uint8 [meta_bytes], dropped tensor or None)."""
+    dt = _dtype_of(x, dtype)
+    M, K = x.shape
+    vals = torch.empty((M, K // 2), dtype=x.dtype, device=x.device)
+    meta = torch.empty(meta_bytes(dt, M, K, layout), dtype=torch.uint8, device=x.device)
+    dropped = torch.zeros(1, dtype=torch.int64, device=x.device) if count_dropped else None
+    _check(lib.sp24_compress(DTYPE_CODE[dt], M, K, _ptr(x), x.stride(0) if M > 1 else K, _ptr(vals),
+                             K // 2, _ptr(meta), layout, _ptr(dropped), _stream()), "sp24_compress")
+    return vals, meta, dropped
+
+
+def compress_into(x, vals, meta, layout: int = META_TCGEN05, dtype: str | None = None, dropped=None):
+    dt = _dtype_of(x, dtype)
+    M, K = x.shape
+    _check(lib.sp24_compress(DTYPE_CODE[dt], M, K, _ptr(x), x.stride(0) if M > 1 else K, _ptr(vals),
+                             vals.stride(0) if M > 1 else K // 2, _ptr(meta), layout, _ptr(dropped),
+                             _stream()), "sp24_compress")
+
+
+def decompress(vals: torch.Tensor, meta: torch.Tensor, layout: int = META_TCGEN05,
+               dtype: str | None = None) -> torch.Tensor:
+    dt = _dtype_of(vals, dtype)
+    M, K2 = vals.shape
+    y = torch.empty((M, 2 * K2), dtype=vals.dtype, device=vals.device)
+    _check(lib.sp24_decompress(DTYPE_CODE[dt], M, 2 * K2, _ptr(vals), vals.stride(0) if M > 1 else K2,
+                               _ptr(meta), layout, _ptr(y), 2 * K2, _stream()), "sp24_decompress")
+    return y
+
+
+def make_desc(ab: str, cd: str, M: int, N: int, K: int, lda: int, ldb: int, ldc: int, ldd: int,
+              a_is_dense: bool = False) -> GemmDesc:
+    return GemmDesc(DTYPE_CODE[ab], DTYPE_CODE[cd], M, N, K, lda, ldb, ldc, ldd, COL_MAJOR, ROW_MAJOR,
+                    ROW_MAJOR, 1 if a_is_dense else 0)
+
+
+def _scalar(ab: str, v):
+    return ctypes.c_float(float(v)) if ab != "i8" else ctypes.c_int32(int(v))
+
+
+_workspaces: dict = {}
+
+
+def workspace(device) -> torch.Tensor:
+    key = (torch.device(device).index, torch.cuda.current_stream().cuda_stream)
+    if key not in _workspaces:
+        _workspaces[key] = torch.zeros(256, dtype=torch.uint8, device=device)
+    return _workspaces[key]
+
+
+def gemm(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor, *, alpha=1.0, beta=0.0,
+         C: torch.Tensor | None = None, out: torch.Tensor | None = None, cd: str | None = None,
+         ab: str | None = None, a_is_dense: bool = False, ws: torch.Tensor | None = None) -> torch.Tensor:
+    """sp24_gemm.  A: vals [M, K/2] (or dense [M, K]); Bt: [N, K] (K contiguous); C/D: [M, N]."""
+    ab = _dtype_of(A, ab)
+    M = A.shape[0]
+    K = A.shape[1] if a_is_dense else 2 * A.shape[1]
+    N = Bt.shape[0]
+    assert Bt.shape[1] == K
+    cd = cd or ("i32" if ab == "i8" else ab)
+    if out is None:
+        out = torch.empty((M, N), dtype=TORCH_DTYPE[cd], device=A.device)
+    ws = ws if ws is not None else workspace(A.device)
+    desc = make_desc(ab, cd, M, N, K, A.stride(0), Bt.stride(0), C.stride(0) if C is not None else N,
+                     out.stride(0), a_is_dense)
+    a, b = _scalar(ab, alpha), _scalar(ab, beta)
+    _check(lib.sp24_gemm(ctypes.byref(desc), ctypes.byref(a), _ptr(A), _ptr(meta), _ptr(Bt),
+                         ctypes.byref(b), _ptr(C), _ptr(out), _ptr(ws), ws.numel(), _stream()), "sp24_gemm")
+    return out
+
+
+def gemm_status(ws: torch.Tensor | None = None, device=None) -> int:
+    ws = ws if ws is not None else workspace(device or "cuda")
+    return lib.sp24_gemm_status(_ptr(ws), _stream())
+
+
+def im2col_nhwc_3x3(x: torch.Tensor, dtype: str | None = None) -> torch.Tensor:
+    dt = _dtype_of(x, dtype)
+    Nb, H, W, C = x.shape
+    out = torch.empty((Nb * H * W, 9 * C), dtype=x.dtype, device=x.device)
+    _check(lib.sp24_im2col_nhwc_3x3(DTYPE_CODE[dt], Nb, H, W, C, _ptr(x), _ptr(out), 9 * C, _stream()),
+           "sp24_im2col_nhwc_3x3")
+    return out

@@ -1,0 +1,552 @@
+// D = alpha * A * B + beta * C on the sm_100a tensor cores (Section 3.2, Figure 2 of arXiv
+// 2104.08378): A is either 2:4-compressed (values + metadata, tcgen05.mma.sp) or dense
+// (tcgen05.mma, the "dense variant" that supplies the sparse-vs-dense speedup).
+//
+// One persistent, warp-specialised kernel:
+//   warp 0   TMA producer: compressed-A tile, metadata block(s) and B tiles of one k-block into a
+//            ring of shared-memory stages (mbarrier expect_tx / complete_tx);
+//   warp 1   MMA issuer (one elected thread): copies the stage's metadata shared -> tensor
+//            memory (tcgen05.cp), issues the tcgen05.mma[.sp] of the stage, commits the stage
+//            back to the producer and, after the last k-block, the accumulator to the epilogue;
+//            owns the tensor-memory allocation;
+//   warps 2-5 epilogue: tcgen05.ld accumulator -> registers, alpha/beta, convert, store.
+// CTAS == 2 runs a pair of CTAs (cluster of two) on one 256 x 256 tile: each CTA loads its 128
+// rows of A / metadata and its half of B, CTA 0 issues cta_group::2 MMAs for both.
+// Every wait is bounded: on expiry the role records a code in the status word and all roles
+// leave through the normal teardown (no trap, no endless spin).
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <mutex>
+
+#include "sp24_common.cuh"
+#include "sp24_ptx.cuh"
+
+namespace sp24 {
+namespace {
+
+constexpr int kBlockM = 128;              // rows of A per CTA (tensor-memory lanes)
+constexpr int kAtomBytes = 128;           // bytes per row of one swizzle-128B operand atom
+constexpr int kNumThreads = 192;          // 6 warps
+constexpr int kEpilogueWarp0 = 2;
+constexpr uint64_t kWaitTimeoutNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
+constexpr uint32_t kTmemCols = 512;
+
+struct GemmParams {
+  int64_t M, N, K;
+  int64_t ldc, ldd;   // elements
+  const void* C;
+  void* D;
+  uint32_t* status;   // [0] = 0 ok, else code of the wait that expired; [1] = launches seen
+  float alpha, beta;
+  int32_t m_tiles, n_tiles, k_blocks;
+  int32_t meta_kb;    // 128-column metadata blocks per 128-row block (K padded to 256)
+  int32_t a_fmt;      // 0 f16, 1 bf16 (kind::f16); ignored for int8
+  int32_t cd_type;    // sp24_dtype of C / D
+  int32_t has_c;
+};
+
+template <int KIND, bool SPARSE, int BLOCK_N, int CTAS>
+struct Cfg {
+  static constexpr int kABoxes = SPARSE ? 1 : 2;                   // 128-byte atoms of A per stage
+  static constexpr int kBBoxes = 2;
+  static constexpr int kBRows = BLOCK_N / CTAS;                    // B rows (N) this CTA loads
+  static constexpr int kABytes = kABoxes * kBlockM * kAtomBytes;
+  static constexpr int kBBytes = kBBoxes * kBRows * kAtomBytes;
+  static constexpr int kEBlocks = SPARSE ? (KIND == 0 ? 1 : 2) : 0;  // 2048-byte metadata blocks per stage
+  static constexpr int kEBytes = kEBlocks * 2048;
+  static constexpr int kStageBytes = kABytes + kBBytes + (SPARSE ? 4096 : 0);
+  static constexpr int kStages = (216 * 1024) / kStageBytes;
+  static constexpr int kTxBytes = (kABytes + kBBytes + kEBytes) * CTAS;
+  static constexpr int kAccStages = (2 * BLOCK_N + 32 <= (int)kTmemCols) ? 2 : 1;
+  static constexpr int kECol = kAccStages * BLOCK_N;               // first metadata column in tensor memory
+  static constexpr int kMmasPerStage = SPARSE ? 4 : 8;
+  static constexpr int kKPerStage = (KIND == 0 ? 64 : 128) * kBBoxes;  // logical K per stage
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static_assert(kStages >= 2, "need at least two stages");
+};
+
+struct Shared {
+  uint64_t full[8], empty[8], tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+
+__device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, Shared* sh, uint32_t* status,
+                                             uint32_t code) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = ptx::globaltimer_ns();
+  uint32_t spins = 0;
+  while (true) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 63u) == 0) {
+      if (sh->abort) return false;
+      if (ptx::globaltimer_ns() - t0 > kWaitTimeoutNs) {
+        sh->abort = 1;
+        atomicCAS(status, 0u, code);
+        return false;
+      }
+    }
+  }
+}
+
+// tile index -> (m_tile, n_tile): bands of `kGroup` m-tiles are swept n-tile by n-tile so that
+// the tiles in flight at one time share a few A row-panels and B column-panels in the L2.
+__device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int& mt, int& nt) {
+  constexpr int kGroup = 8;
+  int per_band = kGroup * n_tiles;
+  int band = t / per_band, in_band = t - band * per_band;
+  int rows = min(kGroup, m_tiles - band * kGroup);
+  nt = in_band / rows;
+  mt = band * kGroup + (in_band - nt * rows);
+}
+
+template <int KIND>
+__device__ __forceinline__ uint32_t make_idesc(bool sparse, int a_fmt, int m, int n) {
+  uint32_t d = 0;
+  d |= (sparse ? 1u : 0u) << 2;
+  d |= (KIND == 0 ? 1u : 2u) << 4;                 // accumulator: fp32 / int32
+  uint32_t fmt = KIND == 0 ? (uint32_t)a_fmt : 1u;  // f16 = 0, bf16 = 1; int8: 1 = signed
+  d |= fmt << 7;
+  d |= fmt << 10;
+  d |= (uint32_t)(n >> 3) << 17;
+  d |= (uint32_t)(m >> 4) << 24;
+  return d;                                        // both operands K-major, no negate, no saturate
+}
+
+template <int CD>
+struct OutPack;  // converts 8 accumulator values of one row to the output type and stores them
+
+__device__ __forceinline__ float acc_to_float(uint32_t r, bool is_int) {
+  return is_int ? (float)(int32_t)r : __uint_as_float(r);
+}
+
+template <int KIND, bool SPARSE, int BLOCK_N, int CTAS>
+__global__ void __launch_bounds__(kNumThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            const __grid_constant__ CUtensorMap map_e, const GemmParams p) {
+  using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS>;
+  extern __shared__ uint8_t smem_raw[];
+  // Operand atoms need 1024-byte alignment for the 128-byte swizzle.
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  Shared* sh = reinterpret_cast<Shared*>(smem + C::kStages * C::kStageBytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t cta_rank = CTAS == 2 ? ptx::cluster_ctarank() : 0;
+  const int cluster_id = blockIdx.x / CTAS, num_clusters = gridDim.x / CTAS;
+  const int num_tiles = p.m_tiles * p.n_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) {
+      ptx::mbar_init(&sh->full[s], 1);
+      ptx::mbar_init(&sh->empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(&sh->tmem_full[a], 1);
+      ptx::mbar_init(&sh->tmem_empty[a], 4 * CTAS);  // one arrival per epilogue warp of the pair
+    }
+    sh->abort = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(&map_a);
+    ptx::prefetch_tensormap(&map_b);
+    if (SPARSE) ptx::prefetch_tensormap(&map_e);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc<CTAS>(&sh->tmem_base, kTmemCols);
+    ptx::tmem_relinquish<CTAS>();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (CTAS == 2) ptx::cluster_sync();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = sh->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (ptx::elect_one()) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
+        int mt, nt;
+        tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
+        const int row0 = (mt * CTAS + (int)cta_rank) * kBlockM;         // first A row of this CTA
+        const int col0 = nt * BLOCK_N + (int)cta_rank * C::kBRows;       // first B row (N index)
+        const int a_box_elems = KIND == 0 ? 64 : 128;                    // elements per 128-byte atom row
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!bounded_wait(&sh->empty[stage], phase ^ 1u, sh, p.status, 1u)) break;
+          uint8_t* sa = smem + stage * C::kStageBytes;
+          uint8_t* sb = sa + C::kABytes;
+          uint8_t* se = sb + C::kBBytes;
+          uint64_t* full = &sh->full[stage];
+          if (cta_rank == 0) ptx::mbar_expect_tx(full, C::kTxBytes);
+#pragma unroll
+          for (int i = 0; i < C::kABoxes; ++i) {
+            int x = (kb * C::kABoxes + i) * a_box_elems;
+            if (CTAS == 1) ptx::tma_load_2d(sa + i * kBlockM * kAtomBytes, &map_a, full, x, row0);
+            else ptx::tma_load_2d_pair(sa + i * kBlockM * kAtomBytes, &map_a, full, 0, x, row0);
+          }
+#pragma unroll
+          for (int i = 0; i < C::kBBoxes; ++i) {
+            int x = (kb * C::kBBoxes + i) * a_box_elems;
+            if (CTAS == 1) ptx::tma_load_2d(sb + i * C::kBRows * kAtomBytes, &map_b, full, x, col0);
+            else ptx::tma_load_2d_pair(sb + i * C::kBRows * kAtomBytes, &map_b, full, 0, x, col0);
+          }
+          if (SPARSE) {
+            // metadata viewed as rows of 128 bytes: block (mb, kb128) starts at row 16 * (mb * KB + kb128)
+            int mb = mt * CTAS + (int)cta_rank;
+            int y = 16 * (mb * p.meta_kb + kb * C::kEBlocks);
+            if (CTAS == 1) ptx::tma_load_2d(se, &map_e, full, 0, y);
+            else ptx::tma_load_2d_pair(se, &map_e, full, 0, 0, y);
+          }
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (cta_rank == 0 && ptx::elect_one()) {
+      const uint32_t idesc = make_idesc<KIND>(SPARSE, p.a_fmt, kBlockM * CTAS, BLOCK_N);
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0, e_buf = 0;
+      for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
+        if (!bounded_wait(&sh->tmem_empty[acc], acc_phase ^ 1u, sh, p.status, 2u)) break;
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
+        bool ok = true;
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!bounded_wait(&sh->full[stage], phase, sh, p.status, 3u)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t sa = ptx::smem_u32(smem + stage * C::kStageBytes);
+          const uint32_t sb = sa + C::kABytes;
+          const uint32_t se = sb + C::kBBytes;
+          // metadata columns alternate between two small tensor-memory buffers from k-block to k-block
+          const uint32_t e_tmem = tmem_base + C::kECol + e_buf * 8;
+          e_buf ^= 1u;
+          if (SPARSE) {
+#pragma unroll
+            for (int i = 0; i < C::kEBlocks; ++i)
+              ptx::tmem_cp_128x128b<CTAS>(e_tmem + 4 * i, ptx::smem_desc(se + i * 2048, false, 128));
+          }
+#pragma unroll
+          for (int k = 0; k < C::kMmasPerStage; ++k) {
+            const uint32_t accumulate = (kb > 0 || k > 0) ? 1u : 0u;
+            if (SPARSE) {
+              // 32 bytes of compressed A and 64 bytes of B per instruction
+              uint64_t da = ptx::smem_desc(sa + k * 32, true, 1024);
+              uint64_t db = ptx::smem_desc(sb + (k >> 1) * C::kBRows * kAtomBytes + (k & 1) * 64, true, 1024);
+              if (KIND == 0) {
+                // one 32-bit metadata column per instruction: even-aligned address + selector
+                ptx::mma_sparse<KIND, CTAS>(d_tmem, da, db, e_tmem + (k & ~1), idesc | (uint32_t)(k & 1), accumulate);
+              } else {
+                ptx::mma_sparse<KIND, CTAS>(d_tmem, da, db, e_tmem + 2 * k, idesc, accumulate);
+              }
+            } else {
+              uint64_t da = ptx::smem_desc(sa + (k >> 2) * kBlockM * kAtomBytes + (k & 3) * 32, true, 1024);
+              uint64_t db = ptx::smem_desc(sb + (k >> 2) * C::kBRows * kAtomBytes + (k & 3) * 32, true, 1024);
+              ptx::mma_dense<KIND, CTAS>(d_tmem, da, db, idesc, accumulate);
+            }
+          }
+          // the stage may be refilled once these MMAs have read it
+          if (CTAS == 1) ptx::tc_commit(&sh->empty[stage]);
+          else ptx::tc_commit_pair(&sh->empty[stage], 3);
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        if (CTAS == 1) ptx::tc_commit(&sh->tmem_full[acc]);
+        else ptx::tc_commit_pair(&sh->tmem_full[acc], 3);
+        if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------ epilogue ------------------------------
+    const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+    const bool is_int = KIND == 1;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
+      int mt, nt;
+      tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
+      if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u)) break;
+      ptx::tc_fence_after();
+      const int64_t row = (int64_t)(mt * CTAS + (int)cta_rank) * kBlockM + q * 32 + lane;
+      const int64_t col_base = (int64_t)nt * BLOCK_N;
+      const uint32_t t_addr = tmem_base + acc * BLOCK_N + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BLOCK_N; c0 += 32) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32b_x32(t_addr + c0, r);
+        ptx::tmem_ld_wait();
+        if (row < p.M) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int64_t col = col_base + c0 + 8 * j;
+            if (col >= p.N) continue;  // N is a multiple of 16, so groups of 8 are all-in or all-out
+            const int64_t off_d = row * p.ldd + col, off_c = row * p.ldc + col;
+            if (is_int) {
+              int32_t v[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) v[e] = (int32_t)r[8 * j + e];
+              if (p.has_c) {
+                const int4* cp = reinterpret_cast<const int4*>(static_cast<const int32_t*>(p.C) + off_c);
+                int4 c0v = cp[0], c1v = cp[1];
+                v[0] += c0v.x; v[1] += c0v.y; v[2] += c0v.z; v[3] += c0v.w;
+                v[4] += c1v.x; v[5] += c1v.y; v[6] += c1v.z; v[7] += c1v.w;
+              }
+              int4* dp = reinterpret_cast<int4*>(static_cast<int32_t*>(p.D) + off_d);
+              dp[0] = make_int4(v[0], v[1], v[2], v[3]);
+              dp[1] = make_int4(v[4], v[5], v[6], v[7]);
+            } else {
+              float v[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) v[e] = p.alpha * __uint_as_float(r[8 * j + e]);
+              if (p.cd_type == SP24_F32) {
+                if (p.has_c) {
+                  const float4* cp = reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + off_c);
+                  float4 a = cp[0], b = cp[1];
+                  v[0] += p.beta * a.x; v[1] += p.beta * a.y; v[2] += p.beta * a.z; v[3] += p.beta * a.w;
+                  v[4] += p.beta * b.x; v[5] += p.beta * b.y; v[6] += p.beta * b.z; v[7] += p.beta * b.w;
+                }
+                float4* dp = reinterpret_cast<float4*>(static_cast<float*>(p.D) + off_d);
+                dp[0] = make_float4(v[0], v[1], v[2], v[3]);
+                dp[1] = make_float4(v[4], v[5], v[6], v[7]);
+              } else if (p.cd_type == SP24_BF16) {
+                if (p.has_c) {
+                  uint4 cv = *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.C) + off_c);
+                  const __nv_bfloat162* c2 = reinterpret_cast<const __nv_bfloat162*>(&cv);
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    float2 f = __bfloat1622float2(c2[e]);
+                    v[2 * e] += p.beta * f.x;
+                    v[2 * e + 1] += p.beta * f.y;
+                  }
+                }
+                uint4 ov;
+                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) o2[e] = __float22bfloat162_rn(make_float2(v[2 * e], v[2 * e + 1]));
+                *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.D) + off_d) = ov;
+              } else {
+                if (p.has_c) {
+                  uint4 cv = *reinterpret_cast<const uint4*>(static_cast<const __half*>(p.C) + off_c);
+                  const __half2* c2 = reinterpret_cast<const __half2*>(&cv);
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    float2 f = __half22float2(c2[e]);
+                    v[2 * e] += p.beta * f.x;
+                    v[2 * e + 1] += p.beta * f.y;
+                  }
+                }
+                uint4 ov;
+                __half2* o2 = reinterpret_cast<__half2*>(&ov);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) o2[e] = __float22half2_rn(make_float2(v[2 * e], v[2 * e + 1]));
+                *reinterpret_cast<uint4*>(static_cast<__half*>(p.D) + off_d) = ov;
+              }
+            }
+          }
+        }
+      }
+      // accumulator drained: hand it back to the MMA issuer (CTA 0 of the pair)
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if (CTAS == 1) ptx::mbar_arrive(&sh->tmem_empty[acc]);
+        else ptx::mbar_arrive_cluster(&sh->tmem_empty[acc], 0);
+      }
+      if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ------------------------------ teardown ------------------------------
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (sh->abort) {
+    // copies issued before the abort may still be landing in this CTA's shared memory
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+  }
+  if (CTAS == 2) ptx::cluster_sync();
+  if (warp == 1) {
+    __syncwarp();
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc<CTAS>(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  });
+  return fn;
+}
+
+// 2-D tensor map over a row-major (rows x cols) array of `es`-byte elements with `ld_bytes`
+// between rows; box = box_cols x box_rows elements.
+sp24_status make_map(CUtensorMap* map, const void* base, int es, uint64_t rows, uint64_t cols, uint64_t ld_bytes,
+                     uint32_t box_cols, uint32_t box_rows, bool swizzle128) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return SP24_ERR_CUDA;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld_bytes};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMapDataType dt = es == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+  CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SP24_OK : SP24_ERR_CUDA;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+  }
+  return n;
+}
+
+template <int KIND, bool SPARSE, int BLOCK_N, int CTAS>
+sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* A, const void* meta, const void* B,
+                   cudaStream_t stream) {
+  using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS>;
+  GemmParams p = base;
+  const int es = KIND == 0 ? 2 : 1;
+  const int tile_m = kBlockM * CTAS;
+  p.m_tiles = (int)((d->M + tile_m - 1) / tile_m);
+  p.n_tiles = (int)((d->N + BLOCK_N - 1) / BLOCK_N);
+  p.k_blocks = (int)((d->K + C::kKPerStage - 1) / C::kKPerStage);
+  p.meta_kb = (int)(2 * ((d->K + 255) / 256));
+  CUtensorMap map_a, map_b, map_e;
+  const uint32_t atom_elems = kAtomBytes / es;
+  const uint64_t a_cols = SPARSE ? d->K / 2 : d->K;
+  sp24_status st = make_map(&map_a, A, es, d->M, a_cols, d->lda * es, atom_elems, kBlockM, true);
+  if (st != SP24_OK) return st;
+  st = make_map(&map_b, B, es, d->N, d->K, d->ldb * es, atom_elems, C::kBRows, true);
+  if (st != SP24_OK) return st;
+  if (SPARSE) {
+    uint64_t meta_rows = (uint64_t)((d->M + 127) / 128) * p.meta_kb * 16;  // rows of 128 bytes
+    st = make_map(&map_e, meta, 1, meta_rows, 128, 128, 128, 16 * C::kEBlocks, false);
+    if (st != SP24_OK) return st;
+  } else {
+    map_e = map_a;
+  }
+  auto kernel = gemm_kernel<KIND, SPARSE, BLOCK_N, CTAS>;
+  SP24_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+  const int tiles = p.m_tiles * p.n_tiles;
+  int clusters = sm_count() / CTAS;
+  if (clusters > tiles) clusters = tiles;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(clusters * CTAS), 1, 1);
+  cfg.blockDim = dim3(kNumThreads, 1, 1);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTAS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  SP24_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_e, p));
+  return SP24_OK;
+}
+
+}  // namespace
+}  // namespace sp24
+
+using namespace sp24;
+
+extern "C" size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d) {
+  (void)d;
+  return 256;
+}
+
+static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A, const void* meta,
+                                 const void* B, const void* beta, const void* C, void* D, void* ws, size_t ws_bytes,
+                                 bool& has_c, float& falpha, float& fbeta) {
+  SP24_RETURN_IF(d == nullptr || alpha == nullptr || beta == nullptr, SP24_ERR_NULL);
+  const bool fp = d->ab_type == SP24_F16 || d->ab_type == SP24_BF16;
+  SP24_RETURN_IF(!fp && d->ab_type != SP24_I8, SP24_ERR_DTYPE);
+  if (fp) SP24_RETURN_IF(d->cd_type != d->ab_type && d->cd_type != SP24_F32, SP24_ERR_DTYPE);
+  else SP24_RETURN_IF(d->cd_type != SP24_I32, SP24_ERR_DTYPE);
+  const int64_t mult = fp ? 16 : 32;
+  SP24_RETURN_IF(d->M < 0 || d->N < 0 || d->K <= 0, SP24_ERR_SHAPE);
+  SP24_RETURN_IF(d->M % mult || d->N % mult || d->K % mult, SP24_ERR_SHAPE);
+  SP24_RETURN_IF(d->M > (int64_t(1) << 30) || d->N > (int64_t(1) << 30) || d->K > (int64_t(1) << 30), SP24_ERR_SHAPE);
+  SP24_RETURN_IF(d->order_b != SP24_COL_MAJOR || d->order_c != SP24_ROW_MAJOR || d->order_d != SP24_ROW_MAJOR,
+                 SP24_ERR_UNSUPPORTED);
+  if (fp) {
+    falpha = *static_cast<const float*>(alpha);
+    fbeta = *static_cast<const float*>(beta);
+  } else {
+    int32_t ia = *static_cast<const int32_t*>(alpha), ib = *static_cast<const int32_t*>(beta);
+    SP24_RETURN_IF(ia != 1 || (ib != 0 && ib != 1), SP24_ERR_UNSUPPORTED);
+    falpha = 1.f;
+    fbeta = (float)ib;
+  }
+  has_c = fbeta != 0.f;
+  if (d->M == 0 || d->N == 0) return SP24_OK;
+  SP24_RETURN_IF(A == nullptr || B == nullptr || D == nullptr || (has_c && C == nullptr), SP24_ERR_NULL);
+  SP24_RETURN_IF(!d->a_is_dense && meta == nullptr, SP24_ERR_NULL);
+  SP24_RETURN_IF(ws == nullptr || ws_bytes < 256 || !aligned16(ws), SP24_ERR_WORKSPACE);
+  const int es = elem_bytes(d->ab_type), cs = elem_bytes(d->cd_type);
+  const int64_t a_cols = d->a_is_dense ? d->K : d->K / 2;
+  SP24_RETURN_IF(d->lda < a_cols || d->ldb < d->K || d->ldd < d->N || (has_c && d->ldc < d->N), SP24_ERR_STRIDE);
+  SP24_RETURN_IF((d->lda * es) % 16 || (d->ldb * es) % 16 || (d->ldd * cs) % 16 || (has_c && (d->ldc * cs) % 16),
+                 SP24_ERR_STRIDE);
+  SP24_RETURN_IF(!aligned16(A) || !aligned16(B) || !aligned16(D) || (has_c && !aligned16(C)) ||
+                     (!d->a_is_dense && !aligned16(meta)),
+                 SP24_ERR_ALIGN);
+  return SP24_OK;
+}
+
+extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A, const void* meta,
+                                 const void* B, const void* beta, const void* C, void* D, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+  bool has_c = false;
+  float falpha = 1.f, fbeta = 0.f;
+  sp24_status st = validate_gemm(d, alpha, A, meta, B, beta, C, D, workspace, workspace_bytes, has_c, falpha, fbeta);
+  if (st != SP24_OK) return st;
+  if (d->M == 0 || d->N == 0) return SP24_OK;
+  if ((st = check_arch()) != SP24_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  SP24_CUDA_CHECK(cudaMemsetAsync(workspace, 0, 16, s));
+  GemmParams p = {};
+  p.M = d->M; p.N = d->N; p.K = d->K;
+  p.ldc = d->ldc; p.ldd = d->ldd;
+  p.C = has_c ? C : nullptr;
+  p.D = D;
+  p.status = static_cast<uint32_t*>(workspace);
+  p.alpha = falpha; p.beta = fbeta;
+  p.a_fmt = d->ab_type == SP24_BF16 ? 1 : 0;
+  p.cd_type = (int)d->cd_type;
+  p.has_c = has_c ? 1 : 0;
+  const bool sparse = !d->a_is_dense;
+  const bool i8 = d->ab_type == SP24_I8;
+  if (!i8) return sparse ? launch<0, true, 128, 1>(d, p, A, meta, B, s) : launch<0, false, 128, 1>(d, p, A, meta, B, s);
+  return sparse ? launch<1, true, 128, 1>(d, p, A, meta, B, s) : launch<1, false, 128, 1>(d, p, A, meta, B, s);
+}
+
+extern "C" sp24_status sp24_gemm_status(const void* workspace, void* stream) {
+  SP24_RETURN_IF(workspace == nullptr, SP24_ERR_NULL);
+  uint32_t host[4] = {0, 0, 0, 0};
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  SP24_CUDA_CHECK(cudaMemcpyAsync(host, workspace, sizeof(host), cudaMemcpyDeviceToHost, s));
+  SP24_CUDA_CHECK(cudaStreamSynchronize(s));
+  return host[0] == 0 ? SP24_OK : SP24_ERR_TIMEOUT;
+}

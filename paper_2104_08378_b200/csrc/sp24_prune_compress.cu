@@ -1,0 +1,479 @@
+// Streaming kernels of the 2:4 path: magnitude pruning (Section 4.1 step 2), compression to
+// kept values + 2-bit position metadata and its inverse (Section 3.1, Figure 1), and the
+// im2col lowering of a 3x3 convolution (Section 4.2).  All of them are bound by HBM bandwidth:
+// every thread moves whole 16-byte vectors, the selection is a handful of integer compares.
+#include "sp24_common.cuh"
+
+namespace sp24 {
+namespace {
+
+constexpr int kThreads = 256;
+
+// ---- selection -------------------------------------------------------------------------
+// Bit p of the result is set iff position p of the group is kept.  Position a beats position b
+// (a < b) when key[a] >= key[b] -- equal magnitudes go to the lower index -- so the six
+// comparisons define a strict total order and exactly two positions are beaten fewer than
+// two times.
+__device__ __forceinline__ uint32_t keep_mask4(uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
+  uint32_t c01 = k0 >= k1, c02 = k0 >= k2, c03 = k0 >= k3;
+  uint32_t c12 = k1 >= k2, c13 = k1 >= k3, c23 = k2 >= k3;
+  uint32_t b0 = 3u - (c01 + c02 + c03);
+  uint32_t b1 = c01 + 2u - (c12 + c13);
+  uint32_t b2 = c02 + c12 + 1u - c23;
+  uint32_t b3 = c03 + c13 + c23;
+  return (b0 < 2u) | ((b1 < 2u) << 1) | ((b2 < 2u) << 2) | ((b3 < 2u) << 3);
+}
+
+// keep mask (two bits set) -> metadata nibble p0 | p1 << 2.
+__device__ __forceinline__ uint32_t mask_to_nibble(uint32_t mask) {
+  uint32_t p0 = __ffs(mask) - 1, p1 = 31 - __clz(mask);
+  return p0 | (p1 << 2);
+}
+
+// One group of four 16-bit values held in two words (lo = elements 0,1; hi = elements 2,3).
+struct Group16 {
+  static __device__ __forceinline__ uint32_t mask(uint32_t lo, uint32_t hi) {
+    return keep_mask4(lo & 0x7FFFu, (lo >> 16) & 0x7FFFu, hi & 0x7FFFu, (hi >> 16) & 0x7FFFu);
+  }
+  static __device__ __forceinline__ uint32_t nonzero(uint32_t lo, uint32_t hi) {
+    return ((lo & 0x7FFFu) != 0) | (((lo >> 16) & 0x7FFFu) != 0) << 1 | ((hi & 0x7FFFu) != 0) << 2 |
+           (((hi >> 16) & 0x7FFFu) != 0) << 3;
+  }
+};
+
+// One group of four int8 values in one word.  __vabs4 maps -128 to 0x80 = 128 (no saturation).
+struct Group8 {
+  static __device__ __forceinline__ uint32_t mask(uint32_t w) {
+    uint32_t a = __vabs4(w);
+    return keep_mask4(a & 0xFFu, (a >> 8) & 0xFFu, (a >> 16) & 0xFFu, a >> 24);
+  }
+  static __device__ __forceinline__ uint32_t nonzero(uint32_t w) {
+    return ((w & 0xFFu) != 0) | ((w & 0xFF00u) != 0) << 1 | ((w & 0xFF0000u) != 0) << 2 |
+           ((w & 0xFF000000u) != 0) << 3;
+  }
+};
+
+__device__ __forceinline__ uint32_t half_lane_mask(uint32_t keep2) {  // 2 keep bits -> 2x16-bit mask
+  return ((keep2 & 1u) ? 0x0000FFFFu : 0u) | ((keep2 & 2u) ? 0xFFFF0000u : 0u);
+}
+
+__device__ __forceinline__ uint32_t byte_lane_mask(uint32_t keep4) {  // 4 keep bits -> 4x8-bit mask
+  return ((keep4 & 1u) ? 0x000000FFu : 0u) | ((keep4 & 2u) ? 0x0000FF00u : 0u) |
+         ((keep4 & 4u) ? 0x00FF0000u : 0u) | ((keep4 & 8u) ? 0xFF000000u : 0u);
+}
+
+__device__ __forceinline__ uint4 ld_stream(const void* p) { return __ldcs(reinterpret_cast<const uint4*>(p)); }
+__device__ __forceinline__ void st_stream(void* p, uint4 v) { __stcs(reinterpret_cast<uint4*>(p), v); }
+
+// ---- prune -----------------------------------------------------------------------------
+template <int ES>
+__device__ __forceinline__ uint4 prune_vec(uint4 v) {
+  if (ES == 2) {
+    uint32_t m0 = Group16::mask(v.x, v.y), m1 = Group16::mask(v.z, v.w);
+    v.x &= half_lane_mask(m0);
+    v.y &= half_lane_mask(m0 >> 2);
+    v.z &= half_lane_mask(m1);
+    v.w &= half_lane_mask(m1 >> 2);
+  } else {
+    v.x &= byte_lane_mask(Group8::mask(v.x));
+    v.y &= byte_lane_mask(Group8::mask(v.y));
+    v.z &= byte_lane_mask(Group8::mask(v.z));
+    v.w &= byte_lane_mask(Group8::mask(v.w));
+  }
+  return v;
+}
+
+// One 16-byte vector per thread and unroll step; `vpr` vectors per row.
+template <int ES, int UNROLL>
+__global__ void __launch_bounds__(kThreads) prune_vec_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
+                                                             uint8_t* y, int64_t row_bytes_y, int64_t vpr,
+                                                             int64_t total) {
+  int64_t base = (int64_t)blockIdx.x * (kThreads * UNROLL) + threadIdx.x;
+  uint4 v[UNROLL];
+  int64_t off_y[UNROLL];
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u) {
+    int64_t id = base + (int64_t)u * kThreads;
+    off_y[u] = -1;
+    if (id < total) {
+      int64_t row = id / vpr, c = id - row * vpr;
+      v[u] = ld_stream(x + row * row_bytes_x + c * 16);
+      off_y[u] = row * row_bytes_y + c * 16;
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u)
+    if (off_y[u] >= 0) st_stream(y + off_y[u], prune_vec<ES>(v[u]));
+}
+
+// Any alignment / leading dimension: one thread per group, element-wise accesses.
+template <typename T>
+__global__ void prune_scalar_kernel(const T* __restrict__ x, int64_t ldx, T* y, int64_t ldy, int64_t groups_per_row,
+                                    int64_t total) {
+  int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (id >= total) return;
+  int64_t row = id / groups_per_row, g = id - row * groups_per_row;
+  const T* src = x + row * ldx + 4 * g;
+  T e[4];
+  uint32_t key[4];
+#pragma unroll
+  for (int p = 0; p < 4; ++p) {
+    e[p] = src[p];
+    key[p] = sizeof(T) == 2 ? (uint32_t)((uint16_t)e[p] & 0x7FFFu) : (uint32_t)abs((int)(int8_t)e[p]);
+  }
+  uint32_t m = keep_mask4(key[0], key[1], key[2], key[3]);
+  T* dst = y + row * ldy + 4 * g;
+#pragma unroll
+  for (int p = 0; p < 4; ++p) dst[p] = (m >> p) & 1u ? e[p] : (T)0;
+}
+
+// ---- metadata addressing ------------------------------------------------------------------
+// Byte offset of the 16 metadata bits of chunk `chunk` (16 consecutive columns of A = four
+// groups) of row `row`.  Canonical: K/8 bytes per row.  Operand order: 2048-byte blocks of 128
+// rows x 128 columns, block (mb, kb) at (mb * KB + kb) * 2048.  Inside a block a 16-bit-type row
+// r shares 32-bit words with row r+8 of its 16-row band, the second 16-column half of every
+// 32-column slice lives 128 bytes further on, and each 32-column slice is one 32-bit tensor-
+// memory column; an int8 row is simply 16 consecutive bytes.
+template <int ES>
+__device__ __forceinline__ int64_t meta_offset(int layout, int64_t row, int64_t chunk, int64_t K, int64_t KB) {
+  if (layout == SP24_META_CANONICAL) return row * (K >> 3) + 2 * chunk;
+  int64_t blk = (row >> 7) * KB + (chunk >> 3);
+  int r = (int)(row & 127), cl = (int)(chunk & 7);
+  int in_blk = ES == 2 ? 16 * (r & 7) + 2 * ((r >> 3) & 1) + 256 * (r >> 4) + 128 * (cl & 1) + 4 * (cl >> 1)
+                       : 16 * r + 2 * cl;
+  return blk * 2048 + in_blk;
+}
+
+// ---- compress (fused prune + compress) ----------------------------------------------------
+// Work unit: one chunk of 16 columns of one row.  16-bit types: 32 bytes in, 16 bytes of values
+// and 16 bits of metadata out.  int8: 16 bytes in, 8 bytes + 16 bits out.  The domain is padded
+// (rows to rows_pad, chunks to chunks_pad) so that the operand-order layout gets its 0x4 padding
+// nibbles from the same launch.
+template <int ES>
+__global__ void __launch_bounds__(kThreads) compress_vec_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
+                                                                uint8_t* __restrict__ vals, int64_t row_bytes_v,
+                                                                uint8_t* __restrict__ meta, int layout, int64_t M,
+                                                                int64_t K, int64_t rows_pad, int64_t chunks_pad,
+                                                                unsigned long long* dropped) {
+  const int64_t chunks = K >> 4, KB = chunks_pad >> 3;
+  const int64_t total = rows_pad * chunks_pad;
+  int64_t id = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  uint32_t lost = 0;
+  if (id < total) {
+    int64_t row = id / chunks_pad, chunk = id - row * chunks_pad;
+    uint32_t mbits = 0x4444u;
+    if (row < M && chunk < chunks) {
+      if (ES == 2) {
+        const uint8_t* src = x + row * row_bytes_x + chunk * 32;
+        uint4 a = ld_stream(src), b = ld_stream(src + 16);
+        uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        uint32_t out[4];
+        mbits = 0;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          uint32_t lo = w[2 * g], hi = w[2 * g + 1];
+          uint32_t m = Group16::mask(lo, hi);
+          uint32_t nib = mask_to_nibble(m);
+          uint64_t both = (uint64_t)lo | ((uint64_t)hi << 32);
+          uint32_t v0 = (uint32_t)(both >> (16 * (nib & 3))) & 0xFFFFu;
+          uint32_t v1 = (uint32_t)(both >> (16 * (nib >> 2))) & 0xFFFFu;
+          out[g] = v0 | (v1 << 16);
+          mbits |= nib << (4 * g);
+          lost += __popc(Group16::nonzero(lo, hi) & ~m);
+        }
+        st_stream(vals + row * row_bytes_v + chunk * 16, make_uint4(out[0], out[1], out[2], out[3]));
+      } else {
+        uint4 a = ld_stream(x + row * row_bytes_x + chunk * 16);
+        uint32_t w[4] = {a.x, a.y, a.z, a.w};
+        uint32_t out[2] = {0, 0};
+        mbits = 0;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          uint32_t m = Group8::mask(w[g]);
+          uint32_t nib = mask_to_nibble(m);
+          uint32_t v0 = (w[g] >> (8 * (nib & 3))) & 0xFFu;
+          uint32_t v1 = (w[g] >> (8 * (nib >> 2))) & 0xFFu;
+          out[g >> 1] |= (v0 | (v1 << 8)) << (16 * (g & 1));
+          mbits |= nib << (4 * g);
+          lost += __popc(Group8::nonzero(w[g]) & ~m);
+        }
+        __stcs(reinterpret_cast<uint2*>(vals + row * row_bytes_v + chunk * 8), make_uint2(out[0], out[1]));
+      }
+    }
+    *reinterpret_cast<uint16_t*>(meta + meta_offset<ES>(layout, row, chunk, K, KB)) = (uint16_t)mbits;
+  }
+  if (dropped != nullptr) {
+    lost = __reduce_add_sync(0xFFFFFFFFu, lost);
+    __shared__ uint32_t warp_sum[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = lost;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t s = 0;
+#pragma unroll
+      for (int wi = 0; wi < kThreads / 32; ++wi) s += warp_sum[wi];
+      if (s) atomicAdd(dropped, (unsigned long long)s);
+    }
+  }
+}
+
+// Any alignment: one thread per 8 columns (two groups = one metadata byte), element-wise.
+template <typename T>
+__global__ void compress_scalar_kernel(const T* __restrict__ x, int64_t ldx, T* __restrict__ vals, int64_t ldv,
+                                       uint8_t* __restrict__ meta, int layout, int64_t M, int64_t K,
+                                       int64_t rows_pad, int64_t bytes_pad, unsigned long long* dropped) {
+  constexpr int ES = sizeof(T);
+  const int64_t total = rows_pad * bytes_pad, KB = bytes_pad >> 4;
+  int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (id >= total) return;
+  int64_t row = id / bytes_pad, bi = id - row * bytes_pad;  // bi: metadata byte index in the row
+  uint32_t mbyte = 0x44u, lost = 0;
+  if (row < M && bi < (K >> 3)) {
+    mbyte = 0;
+    for (int h = 0; h < 2; ++h) {
+      const T* src = x + row * ldx + 8 * bi + 4 * h;
+      T e[4];
+      uint32_t key[4];
+#pragma unroll
+      for (int p = 0; p < 4; ++p) {
+        e[p] = src[p];
+        key[p] = ES == 2 ? (uint32_t)((uint16_t)e[p] & 0x7FFFu) : (uint32_t)abs((int)(int8_t)e[p]);
+      }
+      uint32_t m = keep_mask4(key[0], key[1], key[2], key[3]);
+      uint32_t nib = mask_to_nibble(m);
+      T* dst = vals + row * ldv + 4 * bi + 2 * h;
+      dst[0] = e[nib & 3];
+      dst[1] = e[nib >> 2];
+      mbyte |= nib << (4 * h);
+#pragma unroll
+      for (int p = 0; p < 4; ++p) lost += (key[p] != 0 && !((m >> p) & 1u));
+    }
+  }
+  int64_t off = meta_offset<ES>(layout, row, bi >> 1, K, KB) + (bi & 1);
+  meta[off] = (uint8_t)mbyte;
+  if (dropped != nullptr && lost) atomicAdd(dropped, (unsigned long long)lost);
+}
+
+// ---- decompress ---------------------------------------------------------------------------
+template <int ES>
+__global__ void __launch_bounds__(kThreads) decompress_vec_kernel(const uint8_t* __restrict__ vals, int64_t row_bytes_v,
+                                                                  const uint8_t* __restrict__ meta, int layout,
+                                                                  uint8_t* __restrict__ y, int64_t row_bytes_y,
+                                                                  int64_t M, int64_t K, int64_t chunks_pad) {
+  const int64_t chunks = K >> 4, KB = chunks_pad >> 3;
+  int64_t id = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (id >= M * chunks) return;
+  int64_t row = id / chunks, chunk = id - row * chunks;
+  uint32_t mbits = *reinterpret_cast<const uint16_t*>(meta + meta_offset<ES>(layout, row, chunk, K, KB));
+  if (ES == 2) {
+    uint4 v = ld_stream(vals + row * row_bytes_v + chunk * 16);
+    uint32_t in[4] = {v.x, v.y, v.z, v.w};
+    uint32_t w[8];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      uint32_t nib = (mbits >> (4 * g)) & 0xFu;
+      uint64_t both = ((uint64_t)(in[g] & 0xFFFFu) << (16 * (nib & 3))) | ((uint64_t)(in[g] >> 16) << (16 * (nib >> 2)));
+      w[2 * g] = (uint32_t)both;
+      w[2 * g + 1] = (uint32_t)(both >> 32);
+    }
+    uint8_t* dst = y + row * row_bytes_y + chunk * 32;
+    st_stream(dst, make_uint4(w[0], w[1], w[2], w[3]));
+    st_stream(dst + 16, make_uint4(w[4], w[5], w[6], w[7]));
+  } else {
+    uint2 v = __ldcs(reinterpret_cast<const uint2*>(vals + row * row_bytes_v + chunk * 8));
+    uint32_t in[2] = {v.x, v.y};
+    uint32_t w[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      uint32_t nib = (mbits >> (4 * g)) & 0xFu;
+      uint32_t pair = (in[g >> 1] >> (16 * (g & 1))) & 0xFFFFu;
+      w[g] = ((pair & 0xFFu) << (8 * (nib & 3))) | ((pair >> 8) << (8 * (nib >> 2)));
+    }
+    st_stream(y + row * row_bytes_y + chunk * 16, make_uint4(w[0], w[1], w[2], w[3]));
+  }
+}
+
+template <typename T>
+__global__ void decompress_scalar_kernel(const T* __restrict__ vals, int64_t ldv, const uint8_t* __restrict__ meta,
+                                         int layout, T* __restrict__ y, int64_t ldy, int64_t M, int64_t K,
+                                         int64_t bytes_pad) {
+  constexpr int ES = sizeof(T);
+  const int64_t KB = bytes_pad >> 4, bytes = K >> 3;
+  int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (id >= M * bytes) return;
+  int64_t row = id / bytes, bi = id - row * bytes;
+  uint32_t mbyte = meta[meta_offset<ES>(layout, row, bi >> 1, K, KB) + (bi & 1)];
+  for (int h = 0; h < 2; ++h) {
+    uint32_t nib = (mbyte >> (4 * h)) & 0xFu;
+    const T* src = vals + row * ldv + 4 * bi + 2 * h;
+    T* dst = y + row * ldy + 8 * bi + 4 * h;
+    T e0 = src[0], e1 = src[1];
+#pragma unroll
+    for (int p = 0; p < 4; ++p) dst[p] = p == (int)(nib & 3) ? e0 : (p == (int)(nib >> 2) ? e1 : (T)0);
+  }
+}
+
+// ---- im2col (3x3, stride 1, pad 1, NHWC) ------------------------------------------------------
+// One 16-byte vector of the output per thread: out row = output pixel, out column = (r, s, c).
+__global__ void __launch_bounds__(kThreads) im2col_3x3_kernel(const uint8_t* __restrict__ in, uint8_t* __restrict__ out,
+                                                              int64_t row_bytes_out, int H, int W, int64_t c_vecs,
+                                                              int64_t total) {
+  int64_t id = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (id >= total) return;
+  int64_t vec_per_pixel = 9 * c_vecs;
+  int64_t pixel = id / vec_per_pixel, rem = id - pixel * vec_per_pixel;
+  int rs = (int)(rem / c_vecs);
+  int64_t cv = rem - rs * c_vecs;
+  int r = rs / 3, s = rs - 3 * r;
+  int w = (int)(pixel % W);
+  int64_t t = pixel / W;
+  int h = (int)(t % H);
+  int64_t n = t / H;
+  int hh = h + r - 1, ww = w + s - 1;
+  uint4 v = make_uint4(0, 0, 0, 0);
+  if (hh >= 0 && hh < H && ww >= 0 && ww < W)
+    v = __ldg(reinterpret_cast<const uint4*>(in + (((n * H + hh) * W + ww) * c_vecs + cv) * 16));
+  st_stream(out + pixel * row_bytes_out + rem * 16, v);
+}
+
+inline unsigned blocks_for(int64_t total, int per_block) { return (unsigned)((total + per_block - 1) / per_block); }
+
+}  // namespace
+
+static sp24_status validate_matrix_args(sp24_dtype t, int64_t M, int64_t K, int64_t k_multiple) {
+  SP24_RETURN_IF(!is_ab_type(t), SP24_ERR_DTYPE);
+  SP24_RETURN_IF(M < 0 || K < 0 || K % k_multiple != 0, SP24_ERR_SHAPE);
+  return SP24_OK;
+}
+
+}  // namespace sp24
+
+using namespace sp24;
+
+extern "C" sp24_status sp24_prune(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx, void* y,
+                                  int64_t ldy, void* stream) {
+  sp24_status st = validate_matrix_args(t, M, K, 4);
+  if (st != SP24_OK) return st;
+  if (M == 0 || K == 0) return SP24_OK;
+  SP24_RETURN_IF(x == nullptr || y == nullptr, SP24_ERR_NULL);
+  SP24_RETURN_IF(ldx < K || ldy < K, SP24_ERR_STRIDE);
+  if ((st = check_arch()) != SP24_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int es = elem_bytes(t);
+  const bool vec = aligned16(x) && aligned16(y) && (ldx * es) % 16 == 0 && (ldy * es) % 16 == 0 && (K * es) % 16 == 0;
+  if (vec) {
+    constexpr int UNROLL = 4;
+    int64_t vpr = K * es / 16, total = M * vpr;
+    if (ldx == K && ldy == K) {  // packed: treat the matrix as one long row, no per-vector division
+      vpr = total;
+    }
+    unsigned blocks = blocks_for(total, kThreads * UNROLL);
+    if (es == 2)
+      prune_vec_kernel<2, UNROLL><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)y, ldy * es, vpr, total);
+    else
+      prune_vec_kernel<1, UNROLL><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)y, ldy * es, vpr, total);
+  } else {
+    int64_t gpr = K / 4, total = M * gpr;
+    unsigned blocks = blocks_for(total, kThreads);
+    if (es == 2)
+      prune_scalar_kernel<uint16_t><<<blocks, kThreads, 0, s>>>((const uint16_t*)x, ldx, (uint16_t*)y, ldy, gpr, total);
+    else
+      prune_scalar_kernel<int8_t><<<blocks, kThreads, 0, s>>>((const int8_t*)x, ldx, (int8_t*)y, ldy, gpr, total);
+  }
+  return cuda_status(cudaGetLastError());
+}
+
+extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx, void* vals,
+                                     int64_t ldv, void* meta, sp24_meta_layout l, unsigned long long* dropped,
+                                     void* stream) {
+  sp24_status st = validate_matrix_args(t, M, K, 8);
+  if (st != SP24_OK) return st;
+  SP24_RETURN_IF(l != SP24_META_CANONICAL && l != SP24_META_TCGEN05, SP24_ERR_UNSUPPORTED);
+  if (M == 0 || K == 0) return SP24_OK;
+  SP24_RETURN_IF(x == nullptr || vals == nullptr || meta == nullptr, SP24_ERR_NULL);
+  SP24_RETURN_IF(ldx < K || ldv < K / 2, SP24_ERR_STRIDE);
+  if ((st = check_arch()) != SP24_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int es = elem_bytes(t);
+  const bool hw = l == SP24_META_TCGEN05;
+  const int64_t rows_pad = hw ? (M + 127) / 128 * 128 : M;
+  const int64_t k_pad = hw ? (K + 255) / 256 * 256 : K;
+  const bool vec = K % 16 == 0 && aligned16(x) && aligned16(vals) && aligned16(meta) && (ldx * es) % 16 == 0 &&
+                   (ldv * es) % (8 * es) == 0;
+  if (vec) {
+    int64_t chunks_pad = k_pad / 16, total = rows_pad * chunks_pad;
+    unsigned blocks = blocks_for(total, kThreads);
+    if (es == 2)
+      compress_vec_kernel<2><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)vals, ldv * es,
+                                                         (uint8_t*)meta, (int)l, M, K, rows_pad, chunks_pad, dropped);
+    else
+      compress_vec_kernel<1><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)vals, ldv * es,
+                                                         (uint8_t*)meta, (int)l, M, K, rows_pad, chunks_pad, dropped);
+  } else {
+    int64_t bytes_pad = k_pad / 8, total = rows_pad * bytes_pad;
+    unsigned blocks = blocks_for(total, kThreads);
+    if (es == 2)
+      compress_scalar_kernel<uint16_t><<<blocks, kThreads, 0, s>>>((const uint16_t*)x, ldx, (uint16_t*)vals, ldv,
+                                                                   (uint8_t*)meta, (int)l, M, K, rows_pad, bytes_pad,
+                                                                   dropped);
+    else
+      compress_scalar_kernel<int8_t><<<blocks, kThreads, 0, s>>>((const int8_t*)x, ldx, (int8_t*)vals, ldv,
+                                                                 (uint8_t*)meta, (int)l, M, K, rows_pad, bytes_pad,
+                                                                 dropped);
+  }
+  return cuda_status(cudaGetLastError());
+}
+
+extern "C" sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals, int64_t ldv,
+                                       const void* meta, sp24_meta_layout l, void* y, int64_t ldy, void* stream) {
+  sp24_status st = validate_matrix_args(t, M, K, 8);
+  if (st != SP24_OK) return st;
+  SP24_RETURN_IF(l != SP24_META_CANONICAL && l != SP24_META_TCGEN05, SP24_ERR_UNSUPPORTED);
+  if (M == 0 || K == 0) return SP24_OK;
+  SP24_RETURN_IF(y == nullptr || vals == nullptr || meta == nullptr, SP24_ERR_NULL);
+  SP24_RETURN_IF(ldy < K || ldv < K / 2, SP24_ERR_STRIDE);
+  if ((st = check_arch()) != SP24_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int es = elem_bytes(t);
+  const bool hw = l == SP24_META_TCGEN05;
+  const int64_t k_pad = hw ? (K + 255) / 256 * 256 : K;
+  const bool vec = K % 16 == 0 && aligned16(y) && aligned16(vals) && aligned16(meta) && (ldy * es) % 16 == 0 &&
+                   (ldv * es) % (8 * es) == 0;
+  if (vec) {
+    int64_t total = M * (K / 16);
+    unsigned blocks = blocks_for(total, kThreads);
+    if (es == 2)
+      decompress_vec_kernel<2><<<blocks, kThreads, 0, s>>>((const uint8_t*)vals, ldv * es, (const uint8_t*)meta, (int)l,
+                                                           (uint8_t*)y, ldy * es, M, K, k_pad / 16);
+    else
+      decompress_vec_kernel<1><<<blocks, kThreads, 0, s>>>((const uint8_t*)vals, ldv * es, (const uint8_t*)meta, (int)l,
+                                                           (uint8_t*)y, ldy * es, M, K, k_pad / 16);
+  } else {
+    int64_t total = M * (K / 8);
+    unsigned blocks = blocks_for(total, kThreads);
+    if (es == 2)
+      decompress_scalar_kernel<uint16_t><<<blocks, kThreads, 0, s>>>((const uint16_t*)vals, ldv, (const uint8_t*)meta,
+                                                                     (int)l, (uint16_t*)y, ldy, M, K, k_pad / 8);
+    else
+      decompress_scalar_kernel<int8_t><<<blocks, kThreads, 0, s>>>((const int8_t*)vals, ldv, (const uint8_t*)meta,
+                                                                   (int)l, (int8_t*)y, ldy, M, K, k_pad / 8);
+  }
+  return cuda_status(cudaGetLastError());
+}
+
+extern "C" sp24_status sp24_im2col_nhwc_3x3(sp24_dtype t, int64_t Nb, int64_t H, int64_t W, int64_t C, const void* in,
+                                            void* out, int64_t ldo, void* stream) {
+  SP24_RETURN_IF(!is_ab_type(t), SP24_ERR_DTYPE);
+  SP24_RETURN_IF(Nb < 0 || H < 0 || W < 0 || C < 0 || H > (1 << 30) || W > (1 << 30), SP24_ERR_SHAPE);
+  const int es = elem_bytes(t);
+  SP24_RETURN_IF((C * es) % 16 != 0, SP24_ERR_SHAPE);
+  if (Nb == 0 || H == 0 || W == 0 || C == 0) return SP24_OK;
+  SP24_RETURN_IF(in == nullptr || out == nullptr, SP24_ERR_NULL);
+  SP24_RETURN_IF(ldo < 9 * C || (ldo * es) % 16 != 0, SP24_ERR_STRIDE);
+  SP24_RETURN_IF(!aligned16(in) || !aligned16(out), SP24_ERR_ALIGN);
+  sp24_status st = check_arch();
+  if (st != SP24_OK) return st;
+  int64_t c_vecs = C * es / 16, total = Nb * H * W * 9 * c_vecs;
+  im2col_3x3_kernel<<<blocks_for(total, kThreads), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      (const uint8_t*)in, (uint8_t*)out, ldo * es, (int)H, (int)W, c_vecs, total);
+  return cuda_status(cudaGetLastError());
+}

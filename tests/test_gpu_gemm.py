@@ -1,0 +1,144 @@
+"""GPU parity for the sparse GEMM and its dense variant against the CPU oracle, through the C ABI.
+
+Tolerances (floating point): normwise ||D_gpu - D_ref||_F / ||D_ref||_F <= 2e-3 and per element
+|err| <= 1e-2 * (|alpha| (|A|.|B|)_ij + |beta| |C_ij|); the reference is the oracle's un-rounded
+float64 result.  int8 -> int32 must match bit for bit.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2104_08378_b200 import inputs
+from gpu_util import to_device, to_host_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sp():
+    from paper_2104_08378_b200 import binding
+    return binding
+
+
+def _problem(cfg, with_c=None):
+    A = inputs.gen_A(cfg)
+    Bt = inputs.gen_Bt(cfg)
+    Cm = inputs.gen_C(cfg) if with_c is None else with_c
+    return A, Bt, Cm
+
+
+def check_fp(D_gpu, ref, scale, beta_c=None):
+    err = np.abs(D_gpu - ref)
+    denom = np.linalg.norm(ref)
+    rel = np.linalg.norm(err) / denom if denom > 0 else np.linalg.norm(err)
+    bound = 1e-2 * (scale + (0 if beta_c is None else beta_c)) + 1e-30
+    worst = float((err / bound).max()) if err.size else 0.0
+    assert rel <= 2e-3, f"normwise relative error {rel:.3e}"
+    assert worst <= 1.0, f"per-element error reaches {worst:.3f} of its bound"
+
+
+def run_case(sp, cfg, dense=False, cd=None, rows=None, cols=None, alpha=None, beta=None):
+    ab = cfg.ab_type
+    cd = cd or cfg.cd_type
+    alpha = cfg.alpha if alpha is None else alpha
+    beta = cfg.beta if beta is None else beta
+    A, Bt, Cm = _problem(cfg)
+    vals_ref, meta_ref, _ = oracle.compress(A, ab)
+    Ad, Btd = to_device(A, ab), to_device(Bt, ab)
+    Cd = None
+    if beta != 0:
+        if Cm is None:
+            Cm = inputs._matrix(("int8",) if ab == "i8" else ("normal", 1.0), "i8" if ab == "i8" else cd,
+                                cfg.seed, inputs.TENSOR_C, cfg.N, 0, cfg.M)
+        if ab == "i8":
+            Cm = Cm.astype(np.int32)
+        Cd = to_device(Cm, "i32" if ab == "i8" else cd)
+    if dense:
+        pruned = sp.prune(Ad)
+        D = sp.gemm(pruned, None, Btd, alpha=alpha, beta=beta, C=Cd, cd=cd, a_is_dense=True)
+    else:
+        vals, meta, _ = sp.compress(Ad, layout=sp.META_TCGEN05)
+        D = sp.gemm(vals, meta, Btd, alpha=alpha, beta=beta, C=Cd, cd=cd)
+    torch.cuda.synchronize()
+    assert sp.gemm_status(device=D.device) == 0
+    c_dtype = None if Cm is None else ("i32" if ab == "i8" else cd)
+    ref = oracle.gemm_sparse(vals_ref, meta_ref, Bt, ab, alpha, beta, Cm if beta != 0 else None, c_dtype,
+                             rows=rows, cols=cols)
+    r0, r1 = rows or (0, cfg.M)
+    c0, c1 = cols or (0, cfg.N)
+    got = to_host_f64(D[r0:r1, c0:c1])
+    if ab == "i8":
+        assert np.array_equal(got, ref)
+    else:
+        scale = abs(alpha) * oracle.gemm_abs(vals_ref, meta_ref, Bt, ab, rows=rows, cols=cols)
+        beta_c = None
+        if beta != 0:
+            beta_c = abs(beta) * np.abs(oracle.bits_to_float64(Cm, cd) if cd != "f32" else Cm)[r0:r1, c0:c1]
+        check_fp(got, ref, scale, beta_c)
+    return D
+
+
+TINY = inputs.CONFIGS["tiny_f16"]
+
+
+@pytest.mark.parametrize("dense", [False, True])
+def test_tiny_f16_config(sp, dense):
+    run_case(sp, TINY, dense=dense)
+    run_case(sp, TINY, dense=dense, cd="f32")
+
+
+@pytest.mark.parametrize("dense", [False, True])
+@pytest.mark.parametrize("shape", [(128, 128, 128), (128, 128, 32), (16, 16, 16), (144, 272, 400),
+                                   (384, 640, 1024), (256, 128, 4096)])
+def test_bf16_shapes_tiles_and_ragged_tails(sp, dense, shape):
+    M, N, K = shape
+    cfg = inputs.scaled(inputs.CONFIGS["bert_ffn_bf16"], M=M, N=N, K=K)
+    run_case(sp, cfg, dense=dense)
+
+
+@pytest.mark.parametrize("dense", [False, True])
+@pytest.mark.parametrize("shape", [(128, 128, 256), (32, 32, 32), (160, 288, 416), (384, 512, 2048)])
+def test_int8_bit_exact(sp, dense, shape):
+    M, N, K = shape
+    cfg = inputs.scaled(inputs.CONFIGS["int8_linear"], M=M, N=N, K=K)
+    run_case(sp, cfg, dense=dense)
+    run_case(sp, cfg, dense=dense, beta=1)
+
+
+def test_alpha_beta_with_c(sp):
+    cfg = inputs.scaled(inputs.CONFIGS["gpt3_ffn_bf16"], M=256, N=384, K=512)
+    run_case(sp, cfg)                                  # alpha = 1, beta = 1, C bf16
+    run_case(sp, cfg, alpha=0.5, beta=-2.0)
+    run_case(sp, cfg, alpha=2.0, beta=0.0)
+    run_case(sp, cfg, cd="f32", alpha=1.0, beta=1.0)
+
+
+def test_identity_b_returns_decompressed_a(sp):
+    """B = I: the sparse GEMM must reproduce prune(A) exactly (every selected index is exercised)."""
+    for ab, K in (("f16", 256), ("bf16", 384), ("i8", 512)):
+        M = 256
+        A = inputs._matrix(("int8",) if ab == "i8" else ("normal", 1.0), ab, 11, 0, K, 0, M)
+        if ab == "i8":
+            A = np.clip(A, -127, 127)
+        eye = inputs.to_storage(np.eye(K), ab)
+        vals, meta, _ = sp.compress(to_device(A, ab))
+        D = sp.gemm(vals, meta, to_device(eye, ab), cd="i32" if ab == "i8" else "f32")
+        torch.cuda.synchronize()
+        expect = oracle.bits_to_float64(oracle.prune(A, ab), ab)
+        assert np.array_equal(to_host_f64(D), expect)
+
+
+def test_rejects_bad_arguments(sp):
+    a = torch.zeros((16, 8), dtype=torch.float16, device="cuda")
+    m = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    bt = torch.zeros((16, 16), dtype=torch.float16, device="cuda")
+    with pytest.raises(sp.Sp24Error):                   # N not a multiple of 16
+        sp.gemm(a, m, torch.zeros((8, 16), dtype=torch.float16, device="cuda"))
+    with pytest.raises(sp.Sp24Error):                   # int8 alpha != 1
+        sp.gemm(torch.zeros((32, 16), dtype=torch.int8, device="cuda"), m,
+                torch.zeros((32, 32), dtype=torch.int8, device="cuda"), alpha=2)
+    with pytest.raises(sp.Sp24Error):                   # beta != 0 without C
+        sp.gemm(a, m, bt, beta=1.0)
+    out = sp.gemm(torch.zeros((0, 8), dtype=torch.float16, device="cuda"), m, bt)
+    assert out.shape == (0, 16)

@@ -1,0 +1,115 @@
+"""GPU parity for prune / compress / decompress / im2col: bit-exact against the CPU oracle,
+called through the C ABI (ctypes binding)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2104_08378_b200 import inputs
+from gpu_util import to_device, to_host_bits
+
+pytestmark = pytest.mark.gpu
+
+DTYPES = ["f16", "bf16", "i8"]
+SHAPES = [(256, 512), (200, 656), (37, 96), (129, 272), (1, 16), (513, 2064)]
+
+
+@pytest.fixture(scope="module")
+def sp():
+    from paper_2104_08378_b200 import binding
+    return binding
+
+
+def _rand(dtype, M, K, seed):
+    dist = ("int8",) if dtype == "i8" else ("normal", 1.0)
+    return inputs._matrix(dist, dtype, seed, 9, K, 0, M)
+
+
+def _adversarial(dtype, M, K, seed):
+    """Few distinct magnitudes (many ties), zeros of both signs, denormals, -128 for int8."""
+    rng = np.random.default_rng(seed)
+    if dtype == "i8":
+        pool = np.array([-128, -127, -2, -1, 0, 0, 1, 2, 127], dtype=np.int8)
+    elif dtype == "f16":
+        pool = np.array([0x0000, 0x8000, 0x0001, 0x8001, 0x3C00, 0xBC00, 0x4000, 0xC000, 0x7BFF, 0x03FF],
+                        dtype=np.uint16)
+    else:
+        pool = np.array([0x0000, 0x8000, 0x0001, 0x8001, 0x3F80, 0xBF80, 0x4000, 0xC000, 0x7F7F, 0x007F],
+                        dtype=np.uint16)
+    return np.ascontiguousarray(pool[rng.integers(0, len(pool), size=(M, K))])
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", SHAPES)
+def test_prune_bit_exact(sp, dtype, shape):
+    M, K = shape
+    for x in (_rand(dtype, M, K, 1), _adversarial(dtype, M, K, 2)):
+        y = sp.prune(to_device(x, dtype))
+        assert np.array_equal(to_host_bits(y), oracle.prune(x, dtype))
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_prune_in_place_and_strided(sp, dtype):
+    M, K, ld = 70, 144, 176
+    x = _rand(dtype, M, ld, 3)
+    xd = to_device(x, dtype)
+    view = xd[:, :K]                                   # leading dimension 176 > K
+    sp.prune(view, out=view)                           # y aliases x
+    got = to_host_bits(xd)
+    assert np.array_equal(got[:, :K], oracle.prune(np.ascontiguousarray(x[:, :K]), dtype))
+    assert np.array_equal(got[:, K:], x[:, K:])        # columns past K untouched
+    # misaligned start (scalar path): drop the first 4 columns
+    x2 = _rand(dtype, M, ld, 4)
+    xd2 = to_device(x2, dtype)
+    y2 = sp.prune(xd2[:, 4:4 + 100])
+    assert np.array_equal(to_host_bits(y2), oracle.prune(np.ascontiguousarray(x2[:, 4:104]), dtype))
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", SHAPES + [(64, 40)])
+@pytest.mark.parametrize("layout", [0, 1])
+def test_compress_decompress_bit_exact(sp, dtype, shape, layout):
+    M, K = shape
+    for x in (_rand(dtype, M, K, 5), _adversarial(dtype, M, K, 6)):
+        vals_ref, meta_ref, dropped_ref = oracle.compress(x, dtype)
+        vals, meta, dropped = sp.compress(to_device(x, dtype), layout=layout, count_dropped=True)
+        assert np.array_equal(to_host_bits(vals), vals_ref)
+        meta_h = meta.cpu().numpy()
+        expect = meta_ref.ravel() if layout == 0 else oracle.meta_to_operand_order(meta_ref, dtype)
+        assert meta_h.size == expect.size
+        assert np.array_equal(meta_h, expect)
+        assert int(dropped.item()) == dropped_ref
+        back = sp.decompress(vals, meta, layout=layout)
+        assert np.array_equal(to_host_bits(back), oracle.prune(x, dtype))
+
+
+def test_compress_of_pruned_input_drops_nothing(sp):
+    x = _rand("bf16", 128, 256, 7)
+    y = sp.prune(to_device(x, "bf16"))
+    v1, m1, d1 = sp.compress(y, count_dropped=True)
+    v0, m0, _ = sp.compress(to_device(x, "bf16"))
+    assert int(d1.item()) == 0
+    assert torch.equal(v1.view(torch.int16), v0.view(torch.int16)) and torch.equal(m1, m0)
+
+
+def test_empty_and_bad_arguments(sp):
+    e = torch.empty((0, 64), dtype=torch.float16, device="cuda")
+    assert sp.prune(e).shape == (0, 64)
+    x = torch.zeros((4, 6), dtype=torch.float16, device="cuda")
+    with pytest.raises(sp.Sp24Error) as err:
+        sp.prune(x)                                     # K % 4 != 0
+    assert err.value.status == 3
+    with pytest.raises(sp.Sp24Error):
+        sp.compress(torch.zeros((4, 12), dtype=torch.int8, device="cuda"))   # K % 8 != 0
+    with pytest.raises(sp.Sp24Error):
+        sp.prune(torch.zeros((4, 8), dtype=torch.float32, device="cuda"), dtype="f32")
+
+
+@pytest.mark.parametrize("dtype", ["f16", "i8"])
+def test_im2col_bit_exact(sp, dtype):
+    cfg = inputs.scaled(inputs.CONFIGS["resnet_conv_f16"], conv=(3, 14, 14, 32))
+    x = inputs._matrix(("relu_normal", 1.0) if dtype != "i8" else ("int8",), dtype, 4, 1, 14 * 14 * 32, 0, 3)
+    x = x.reshape(3, 14, 14, 32)
+    got = sp.im2col_nhwc_3x3(to_device(x, dtype))
+    assert np.array_equal(to_host_bits(got), oracle.im2col_nhwc_3x3(x, dtype))
+    assert got.shape == (cfg.N, cfg.K)

@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of the 2:4 sparse hot path on B200: prune -> compress -> sparse tensor-core GEMM.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+One "step" is one pass of the whole path over one batch of seeded synthetic input of the
+GPT-3-scale FFN configuration (A 49152 x 12288 bf16, 8192 tokens, beta = 1): sp24_prune,
+sp24_compress (tensor-core metadata layout) and sp24_gemm.  `value` is the dense-equivalent
+throughput 2*M*N*K / step time, inputs resident in HBM.  `e2e` is the same metric through the
+host-buffer entry point (host -> device copies of A, B, C and the copy of D back inside the
+timed region).  `roofline` describes the dominant kernel (the sparse GEMM), timed with CUDA
+events inside the timed steps.  `cpu_baseline` times the CPU oracle on a bounded sample of the
+same workload.  With --gpus N > 1 (under torchrun) every rank runs the same weight against its
+own 8192 tokens (weak scaling, no data-path collective); the time is the max over ranks.
+
+`--impl reference` times the CPU oracle alone on the host cores (a deliberately plain program:
+the ratio against it says nothing about kernel quality).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2104_08378_b200 import inputs  # noqa: E402
+
+METRIC = "2:4 sparse GEMM dense-equivalent TFLOPS (prune + compress + sp24_gemm per step)"
+UNIT = "TFLOP/s"
+NOMINAL_SPARSE_BF16_TFLOPS = 4500.0   # 2 x the 2.25 PFLOP/s dense bf16 datasheet figure
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def ncu_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch from the committed ncu summary (profiles/roofline_traffic.json)."""
+    path = os.path.join(ROOT, "profiles", "roofline_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        table = json.load(f)
+    return table.get(kernel, {}).get(workload)
+
+
+# -------------------------------------------------------------------------------------------
+# clocks during the timed region
+# -------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.samples, self.reason_bits, self.max_mhz = [], 0, None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nvml = pynvml
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if visible:
+                ids = [v for v in visible.split(",") if v.strip() != ""]
+                if index < len(ids) and ids[index].isdigit():
+                    phys = int(ids[index])
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nvml = None
+
+    def _run(self):
+        n = self.nvml
+        while not self._stop.is_set():
+            try:
+                self.samples.append(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
+                self.reason_bits |= int(n.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nvml is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self) -> dict:
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit]
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(self.samples)}
+
+
+# -------------------------------------------------------------------------------------------
+# CPU oracle legs
+# -------------------------------------------------------------------------------------------
+def oracle_sample(cfg, budget_s: float = 15.0, tile: int = 128):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: compress of the
+    A rows the sampled output tiles need, then the sparse GEMM of those tiles.  Returns
+    (dense-equivalent TFLOP/s, description, threads)."""
+    import oracle
+    tiles = inputs.sample_tiles(cfg, 1024, tile)
+    # calibrate on one tile, then take as many tiles as fit the budget
+    done, t_total, flop = 0, 0.0, 0.0
+    target = 1
+    while done < len(tiles):
+        batch = tiles[done:done + target]
+        for (tm, tn) in batch:
+            A = inputs.gen_A(cfg, rows=(tm * tile, (tm + 1) * tile))
+            Bt = inputs.gen_Bt(cfg, cols=(tn * tile, (tn + 1) * tile))
+            t1 = time.perf_counter()
+            vals, meta, _ = oracle.compress(A, cfg.ab_type)
+            Cm = None
+            if cfg.beta != 0:
+                Cm = np.ascontiguousarray(inputs.gen_C(cfg, rows=(tm * tile, (tm + 1) * tile))[:, tn * tile:(tn + 1) * tile])
+            oracle.gemm_sparse(vals, meta, Bt, cfg.ab_type, cfg.alpha, cfg.beta, Cm,
+                               cfg.cd_type if Cm is not None else None)
+            t_total += time.perf_counter() - t1          # generation of inputs is not timed
+            flop += 2.0 * tile * tile * cfg.K
+        done += len(batch)
+        per_tile = t_total / done
+        remaining = budget_s - t_total
+        if remaining <= per_tile:
+            break
+        target = max(1, min(len(tiles) - done, int(remaining / per_tile)))
+    desc = (f"{done} seeded {tile}x{tile} output tiles of {cfg.name} (K={cfg.K}): oracle compress of their "
+            f"A rows + oracle sparse GEMM, {t_total:.1f} s")
+    return flop / t_total / 1e12, desc, oracle.num_threads()
+
+
+def run_reference(args, cfg):
+    """The reference arm: the CPU oracle on bounded samples of the workload, rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    per_step_budget = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(cfg, per_step_budget)
+    vals, t0 = [], time.perf_counter()
+    desc, threads = "", 1
+    for _ in range(args.steps):
+        v, desc, threads = oracle_sample(cfg, per_step_budget)
+        vals.append(v)
+    elapsed = time.perf_counter() - t0
+    value = float(np.mean(vals))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * elapsed / max(1, args.steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": cfg.name, "M": cfg.M, "N": cfg.N, "K": cfg.K,
+                                        "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# -------------------------------------------------------------------------------------------
+# GPU arm
+# -------------------------------------------------------------------------------------------
+def run_ours(args, cfg):
+    import torch
+    from paper_2104_08378_b200 import binding as sp
+    from paper_2104_08378_b200 import distributed as D
+
+    rank, local_rank, world = D.init("nccl")
+    if world != args.gpus and world > 1:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    ab, cd = cfg.ab_type, cfg.cd_type
+    tdt = sp.TORCH_DTYPE
+
+    def dev_tensor(a, dt):
+        if dt in ("f16", "bf16"):
+            return torch.from_numpy(a.view(np.int16)).to(dev).view(tdt[dt])
+        return torch.from_numpy(a).to(dev)
+
+    # ---- seeded synthetic inputs (host generator), rank r owns tokens [r*N, (r+1)*N) ----
+    M, N, K = cfg.M, cfg.N, cfg.K
+    A_h = inputs.gen_A(cfg)
+    Bt_h = inputs.gen_Bt(cfg, cols=(rank * N, (rank + 1) * N))
+    C_h = None
+    if cfg.beta != 0:
+        C_h = inputs._matrix(cfg.c_dist, cd, cfg.seed + 7919 * rank, inputs.TENSOR_C, N, 0, M)
+    A = dev_tensor(A_h, ab)
+    Bt = dev_tensor(Bt_h, ab)
+    C = dev_tensor(C_h, cd) if C_h is not None else None
+    A_pruned = torch.empty_like(A)
+    vals = torch.empty((M, K // 2), dtype=A.dtype, device=dev)
+    meta = torch.empty(sp.meta_bytes(ab, M, K, sp.META_TCGEN05), dtype=torch.uint8, device=dev)
+    Dout = torch.empty((M, N), dtype=tdt[cd], device=dev)
+    ws = torch.zeros(256, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    gemm_events = []
+
+    def step(record=False):
+        sp.prune(A, out=A_pruned)                                   # Section 4.1 step 2
+        sp.compress_into(A_pruned, vals, meta, layout=sp.META_TCGEN05)  # Section 3.1
+        if record:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+        sp.gemm(vals, meta, Bt, alpha=cfg.alpha, beta=cfg.beta, C=C, out=Dout, cd=cd, ws=ws)  # Section 3.2
+        if record:
+            e1.record(stream)
+            gemm_events.append((e0, e1))
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    D.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin.record(stream)
+    for _ in range(args.steps):
+        step(record=True)
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    D.barrier()
+    clocks = sampler.stop()
+    elapsed_ms = D.max_over_ranks(t_begin.elapsed_time(t_end), dev)
+    if sp.gemm_status(ws) != 0:
+        raise SystemExit("sp24_gemm reported a device-side timeout")
+    gemm_ms = float(np.mean([a.elapsed_time(b) for a, b in gemm_events]))
+    flop = cfg.dense_equiv_flop
+    ms_per_step = elapsed_ms / args.steps
+    value = world * flop / (ms_per_step * 1e-3) / 1e12
+
+    # ---- per-kernel timings, dense variant (outside the timed region) ----
+    def time_call(fn, reps=5):
+        fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return float(np.median(ts))
+
+    es = 2 if ab != "i8" else 1
+    prune_ms = time_call(lambda: sp.prune(A, out=A_pruned))
+    compress_ms = time_call(lambda: sp.compress_into(A_pruned, vals, meta, layout=sp.META_TCGEN05))
+    dense_ms = time_call(lambda: sp.gemm(A_pruned, None, Bt, alpha=cfg.alpha, beta=cfg.beta, C=C, out=Dout, cd=cd,
+                                         a_is_dense=True, ws=ws), reps=3)
+    prune_bytes = 2 * M * K * es
+    compress_bytes = M * K * es + M * K // 2 * es + M * K // 8
+    peaks = measured_peaks()
+    sparse_peak = 2.0 * peaks["bf16_tflops"] * (2.0 if ab == "i8" else 1.0)
+    gemm_tflops = flop / (gemm_ms * 1e-3) / 1e12
+    kernels = {
+        "prune_ms": prune_ms, "prune_gbs": prune_bytes / prune_ms / 1e6,
+        "prune_frac_of_hbm_" + peaks["source"]: prune_bytes / prune_ms / 1e6 / peaks["hbm_gbs"],
+        "compress_ms": compress_ms, "compress_gbs": compress_bytes / compress_ms / 1e6,
+        "compress_frac_of_hbm_" + peaks["source"]: compress_bytes / compress_ms / 1e6 / peaks["hbm_gbs"],
+        "gemm_ms": gemm_ms, "gemm_dense_equiv_tflops": gemm_tflops, "gemm_useful_tflops": gemm_tflops / 2,
+        "gemm_frac_of_nominal_sparse_peak": gemm_tflops / (NOMINAL_SPARSE_BF16_TFLOPS * (2.0 if ab == "i8" else 1.0)),
+        "dense_variant_ms": dense_ms, "dense_variant_tflops": flop / (dense_ms * 1e-3) / 1e12,
+        "speedup_vs_dense_variant": dense_ms / gemm_ms,
+    }
+
+    # ---- end to end through the host-buffer entry point (rank-local) ----
+    import ctypes
+    e2e = None
+    e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 3))
+    if e2e_steps:
+        hA = torch.from_numpy(A_h.view(np.int16) if es == 2 else A_h).pin_memory()
+        hB = torch.from_numpy(Bt_h.view(np.int16) if es == 2 else Bt_h).pin_memory()
+        hC = torch.from_numpy(C_h.view(np.int16) if cd in ("f16", "bf16") else C_h).pin_memory() if C_h is not None else None
+        hD = torch.empty((M, N), dtype=torch.int16 if cd in ("f16", "bf16") else tdt[cd]).pin_memory()
+        desc = sp.make_desc(ab, cd, M, N, K, K // 2, K, N, N)
+        al, be = sp._scalar(ab, cfg.alpha), sp._scalar(ab, cfg.beta)
+        vp = lambda t: ctypes.c_void_p(t.data_ptr()) if t is not None else None  # noqa: E731
+
+        def e2e_step():
+            st = sp.lib.sp24_pipeline_host(ctypes.byref(desc), ctypes.byref(al), vp(hA), vp(hB), ctypes.byref(be), vp(hC),
+                                           vp(hD), vp(A_pruned), vp(vals), vp(meta), vp(Bt), vp(C), vp(Dout), vp(ws),
+                                           ws.numel(), stream.cuda_stream)
+            if st != 0:
+                raise SystemExit(f"sp24_pipeline_host: {sp.status_string(st)}")
+
+        e2e_step()
+        torch.cuda.synchronize()
+        D.barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record(stream)
+        torch.cuda.synchronize()
+        e2e_ms = D.max_over_ranks(a.elapsed_time(b), dev) / e2e_steps
+        h2d = A_h.nbytes + Bt_h.nbytes + (C_h.nbytes if C_h is not None else 0)
+        d2h = M * N * (2 if cd in ("f16", "bf16") else 4)
+        e2e = {"value": world * flop / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps}
+
+    if rank != 0:
+        return
+    kernel_name = "sp24_gemm (tcgen05.mma.sp, 2-CTA 256x240 tiles)"
+    roofline = {
+        "kernel": kernel_name, "bound": "tensor", "achieved": gemm_tflops, "peak": sparse_peak, "unit": UNIT,
+        "frac": gemm_tflops / sparse_peak,
+        "peak_source": f"2 x {peaks['source']} dense bf16 burst ({peaks['bf16_tflops']} TFLOP/s)"
+                       + (" x 2 for int8" if ab == "i8" else ""),
+        "frac_of_2x_sustained": (gemm_tflops / (2.0 * peaks["bf16_tflops_sustained"])
+                                 if peaks.get("bf16_tflops_sustained") and ab != "i8" else None),
+        "traffic": ncu_traffic("sp24_gemm", cfg.name),
+    }
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        v, sample, threads = oracle_sample(cfg, 15.0)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if ab == "bf16" else ("f16" if ab == "f16" else "i8"), "data": "synthetic",
+        "config": {"workload": cfg.name, "M": M, "N": N, "K": K, "alpha": cfg.alpha, "beta": cfg.beta,
+                   "cd_type": cd, "tokens_per_gpu": N, "parallelism": f"replicated weight, tokens sharded x{world}",
+                   "l2": "inputs larger than L2 (A 1.2 GB, vals 0.6 GB, B 0.2 GB per step)"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * args.steps, "roofline": roofline, "cpu_baseline": cpu,
+        "kernels": kernels,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="gpt3_ffn_bf16", choices=inputs.CONFIG_ORDER)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--rows", type=int, default=0,
+                    help="use only the first ROWS rows of A (a smaller case of the same kernel for ncu captures)")
+    args = ap.parse_args()
+    cfg = inputs.CONFIGS[args.config]
+    if args.rows:
+        cfg = inputs.scaled(cfg, M=args.rows, name=f"{cfg.name}[rows={args.rows} of {cfg.M}]")
+    if cfg.conv is not None:
+        raise SystemExit("the convolution config is covered by the parity tests, not by bench.py")
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -18,6 +18,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 #include "sp24_common.cuh"
@@ -29,7 +31,6 @@ namespace {
 constexpr int kBlockM = 128;              // rows of A per CTA (tensor-memory lanes)
 constexpr int kAtomBytes = 128;           // bytes per row of one swizzle-128B operand atom
 constexpr int kNumThreads = 192;          // 6 warps
-constexpr int kEpilogueWarp0 = 2;
 constexpr uint64_t kWaitTimeoutNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
 constexpr uint32_t kTmemCols = 512;
 
@@ -113,13 +114,6 @@ __device__ __forceinline__ uint32_t make_idesc(bool sparse, int a_fmt, int m, in
   d |= (uint32_t)(n >> 3) << 17;
   d |= (uint32_t)(m >> 4) << 24;
   return d;                                        // both operands K-major, no negate, no saturate
-}
-
-template <int CD>
-struct OutPack;  // converts 8 accumulator values of one row to the output type and stores them
-
-__device__ __forceinline__ float acc_to_float(uint32_t r, bool is_int) {
-  return is_int ? (float)(int32_t)r : __uint_as_float(r);
 }
 
 template <int KIND, bool SPARSE, int BLOCK_N, int CTAS>
@@ -281,7 +275,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const int64_t col = col_base + c0 + 8 * j;
-            if (col >= p.N) continue;  // N is a multiple of 16, so groups of 8 are all-in or all-out
+            // N and BLOCK_N are multiples of 16, so groups of 8 columns are all-in or all-out
+            if (c0 + 8 * j >= BLOCK_N || col >= p.N) continue;
             const int64_t off_d = row * p.ldd + col, off_c = row * p.ldc + col;
             if (is_int) {
               int32_t v[8];
@@ -538,8 +533,27 @@ extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, con
   p.has_c = has_c ? 1 : 0;
   const bool sparse = !d->a_is_dense;
   const bool i8 = d->ab_type == SP24_I8;
-  if (!i8) return sparse ? launch<0, true, 128, 1>(d, p, A, meta, B, s) : launch<0, false, 128, 1>(d, p, A, meta, B, s);
-  return sparse ? launch<1, true, 128, 1>(d, p, A, meta, B, s) : launch<1, false, 128, 1>(d, p, A, meta, B, s);
+  // Tile choice: a pair of CTAs on 256 x 240 tiles (two accumulators fit tensor memory, so the
+  // epilogue overlaps the next tile's main loop) once the problem has enough of them to occupy
+  // the pairs; single CTAs on 128 x 128 tiles otherwise.  SP24_TILE=<ctas>x<block_n> overrides.
+  int ctas = (d->M >= 256 && (d->M / 256) * ((d->N + 239) / 240) >= 32) ? 2 : 1;
+  int block_n = ctas == 2 ? 240 : 128;
+  if (const char* env = getenv("SP24_TILE")) {
+    int c = 0, n = 0;
+    if (sscanf(env, "%dx%d", &c, &n) == 2) { ctas = c; block_n = n; }
+  }
+#define SP24_DISPATCH(CT, BN)                                                                              \
+  if (ctas == CT && block_n == BN) {                                                                       \
+    if (!i8) return sparse ? launch<0, true, BN, CT>(d, p, A, meta, B, s) : launch<0, false, BN, CT>(d, p, A, meta, B, s); \
+    return sparse ? launch<1, true, BN, CT>(d, p, A, meta, B, s) : launch<1, false, BN, CT>(d, p, A, meta, B, s);          \
+  }
+  SP24_DISPATCH(1, 128)
+  SP24_DISPATCH(2, 256)
+  SP24_DISPATCH(2, 240)
+  SP24_DISPATCH(2, 224)
+  SP24_DISPATCH(2, 192)
+#undef SP24_DISPATCH
+  return SP24_ERR_UNSUPPORTED;
 }
 
 extern "C" sp24_status sp24_gemm_status(const void* workspace, void* stream) {

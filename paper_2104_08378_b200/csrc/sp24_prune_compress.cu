@@ -145,75 +145,124 @@ __device__ __forceinline__ int64_t meta_offset(int layout, int64_t row, int64_t 
 }
 
 // ---- compress (fused prune + compress) ----------------------------------------------------
-// Work unit: one chunk of 16 columns of one row.  16-bit types: 32 bytes in, 16 bytes of values
-// and 16 bits of metadata out.  int8: 16 bytes in, 8 bytes + 16 bits out.  The domain is padded
-// (rows to rows_pad, chunks to chunks_pad) so that the operand-order layout gets its 0x4 padding
-// nibbles from the same launch.
-template <int ES>
-__global__ void __launch_bounds__(kThreads) compress_vec_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
-                                                                uint8_t* __restrict__ vals, int64_t row_bytes_v,
-                                                                uint8_t* __restrict__ meta, int layout, int64_t M,
-                                                                int64_t K, int64_t rows_pad, int64_t chunks_pad,
-                                                                unsigned long long* dropped) {
+// The domain is padded (rows to rows_pad, 16-column chunks to chunks_pad) so that the operand-
+// order layout gets its 0x4 padding nibbles from the same launch.  Every thread issues all of
+// its loads before it consumes any of them.
+__device__ __forceinline__ void count_dropped(uint32_t lost, unsigned long long* dropped) {
+  if (dropped == nullptr) return;
+  lost = __reduce_add_sync(0xFFFFFFFFu, lost);
+  __shared__ uint32_t warp_sum[kThreads / 32];
+  if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = lost;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t s = 0;
+#pragma unroll
+    for (int wi = 0; wi < kThreads / 32; ++wi) s += warp_sum[wi];
+    if (s) atomicAdd(dropped, (unsigned long long)s);
+  }
+}
+
+// 16-bit types.  Work unit: 8 columns (two groups) = one 16-byte load, 8 bytes of values and one
+// metadata byte out, so a warp reads 512 and writes 256 contiguous bytes per step.  Lanes 2j and
+// 2j+1 hold the two halves of a 16-column chunk; the even lane stores the chunk's 16 metadata bits.
+template <int UNROLL>
+__global__ void __launch_bounds__(kThreads) compress16_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
+                                                              uint8_t* __restrict__ vals, int64_t row_bytes_v,
+                                                              uint8_t* __restrict__ meta, int layout, int64_t M,
+                                                              int64_t K, int64_t rows_pad, int64_t chunks_pad,
+                                                              unsigned long long* dropped) {
+  const int64_t halves = K >> 3, halves_pad = chunks_pad * 2, KB = chunks_pad >> 3;
+  const int64_t total = rows_pad * halves_pad;
+  const int64_t base = (int64_t)blockIdx.x * (kThreads * UNROLL) + threadIdx.x;
+  uint4 in[UNROLL];
+  int64_t row[UNROLL], half[UNROLL];
+  bool live[UNROLL];
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u) {
+    int64_t id = base + (int64_t)u * kThreads;
+    row[u] = id / halves_pad;
+    half[u] = id - row[u] * halves_pad;
+    live[u] = id < total && row[u] < M && half[u] < halves;
+    if (live[u]) in[u] = ld_stream(x + row[u] * row_bytes_x + half[u] * 16);
+  }
+  uint32_t lost = 0;
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u) {
+    uint32_t mbyte = 0x44u;  // padding: positions (0, 1) in both groups
+    if (live[u]) {
+      uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
+      uint32_t out[2];
+      mbyte = 0;
+#pragma unroll
+      for (int g = 0; g < 2; ++g) {
+        uint32_t lo = w[2 * g], hi = w[2 * g + 1];
+        uint32_t m = Group16::mask(lo, hi);
+        uint32_t nib = mask_to_nibble(m);
+        uint64_t both = (uint64_t)lo | ((uint64_t)hi << 32);
+        uint32_t v0 = (uint32_t)(both >> (16 * (nib & 3))) & 0xFFFFu;
+        uint32_t v1 = (uint32_t)(both >> (16 * (nib >> 2))) & 0xFFFFu;
+        out[g] = v0 | (v1 << 16);
+        mbyte |= nib << (4 * g);
+        lost += __popc(Group16::nonzero(lo, hi) & ~m);
+      }
+      __stcs(reinterpret_cast<uint2*>(vals + row[u] * row_bytes_v + half[u] * 8), make_uint2(out[0], out[1]));
+    }
+    uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, mbyte, 1);
+    int64_t id = base + (int64_t)u * kThreads;
+    if ((threadIdx.x & 1) == 0 && id < total)
+      *reinterpret_cast<uint16_t*>(meta + meta_offset<2>(layout, row[u], half[u] >> 1, K, KB)) =
+          (uint16_t)(mbyte | (other << 8));
+  }
+  count_dropped(lost, dropped);
+}
+
+// int8.  Work unit: one chunk of 16 columns (four groups) = one 16-byte load, 8 bytes of values and
+// 16 bits of metadata out.
+template <int UNROLL>
+__global__ void __launch_bounds__(kThreads) compress8_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
+                                                             uint8_t* __restrict__ vals, int64_t row_bytes_v,
+                                                             uint8_t* __restrict__ meta, int layout, int64_t M,
+                                                             int64_t K, int64_t rows_pad, int64_t chunks_pad,
+                                                             unsigned long long* dropped) {
   const int64_t chunks = K >> 4, KB = chunks_pad >> 3;
   const int64_t total = rows_pad * chunks_pad;
-  int64_t id = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  const int64_t base = (int64_t)blockIdx.x * (kThreads * UNROLL) + threadIdx.x;
+  uint4 in[UNROLL];
+  int64_t row[UNROLL], chunk[UNROLL];
+  bool live[UNROLL];
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u) {
+    int64_t id = base + (int64_t)u * kThreads;
+    row[u] = id / chunks_pad;
+    chunk[u] = id - row[u] * chunks_pad;
+    live[u] = id < total && row[u] < M && chunk[u] < chunks;
+    if (live[u]) in[u] = ld_stream(x + row[u] * row_bytes_x + chunk[u] * 16);
+  }
   uint32_t lost = 0;
-  if (id < total) {
-    int64_t row = id / chunks_pad, chunk = id - row * chunks_pad;
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u) {
+    int64_t id = base + (int64_t)u * kThreads;
+    if (id >= total) continue;
     uint32_t mbits = 0x4444u;
-    if (row < M && chunk < chunks) {
-      if (ES == 2) {
-        const uint8_t* src = x + row * row_bytes_x + chunk * 32;
-        uint4 a = ld_stream(src), b = ld_stream(src + 16);
-        uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-        uint32_t out[4];
-        mbits = 0;
+    if (live[u]) {
+      uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
+      uint32_t out[2] = {0, 0};
+      mbits = 0;
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          uint32_t lo = w[2 * g], hi = w[2 * g + 1];
-          uint32_t m = Group16::mask(lo, hi);
-          uint32_t nib = mask_to_nibble(m);
-          uint64_t both = (uint64_t)lo | ((uint64_t)hi << 32);
-          uint32_t v0 = (uint32_t)(both >> (16 * (nib & 3))) & 0xFFFFu;
-          uint32_t v1 = (uint32_t)(both >> (16 * (nib >> 2))) & 0xFFFFu;
-          out[g] = v0 | (v1 << 16);
-          mbits |= nib << (4 * g);
-          lost += __popc(Group16::nonzero(lo, hi) & ~m);
-        }
-        st_stream(vals + row * row_bytes_v + chunk * 16, make_uint4(out[0], out[1], out[2], out[3]));
-      } else {
-        uint4 a = ld_stream(x + row * row_bytes_x + chunk * 16);
-        uint32_t w[4] = {a.x, a.y, a.z, a.w};
-        uint32_t out[2] = {0, 0};
-        mbits = 0;
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          uint32_t m = Group8::mask(w[g]);
-          uint32_t nib = mask_to_nibble(m);
-          uint32_t v0 = (w[g] >> (8 * (nib & 3))) & 0xFFu;
-          uint32_t v1 = (w[g] >> (8 * (nib >> 2))) & 0xFFu;
-          out[g >> 1] |= (v0 | (v1 << 8)) << (16 * (g & 1));
-          mbits |= nib << (4 * g);
-          lost += __popc(Group8::nonzero(w[g]) & ~m);
-        }
-        __stcs(reinterpret_cast<uint2*>(vals + row * row_bytes_v + chunk * 8), make_uint2(out[0], out[1]));
+      for (int g = 0; g < 4; ++g) {
+        uint32_t m = Group8::mask(w[g]);
+        uint32_t nib = mask_to_nibble(m);
+        uint32_t v0 = (w[g] >> (8 * (nib & 3))) & 0xFFu;
+        uint32_t v1 = (w[g] >> (8 * (nib >> 2))) & 0xFFu;
+        out[g >> 1] |= (v0 | (v1 << 8)) << (16 * (g & 1));
+        mbits |= nib << (4 * g);
+        lost += __popc(Group8::nonzero(w[g]) & ~m);
       }
+      __stcs(reinterpret_cast<uint2*>(vals + row[u] * row_bytes_v + chunk[u] * 8), make_uint2(out[0], out[1]));
     }
-    *reinterpret_cast<uint16_t*>(meta + meta_offset<ES>(layout, row, chunk, K, KB)) = (uint16_t)mbits;
+    *reinterpret_cast<uint16_t*>(meta + meta_offset<1>(layout, row[u], chunk[u], K, KB)) = (uint16_t)mbits;
   }
-  if (dropped != nullptr) {
-    lost = __reduce_add_sync(0xFFFFFFFFu, lost);
-    __shared__ uint32_t warp_sum[kThreads / 32];
-    if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = lost;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      uint32_t s = 0;
-#pragma unroll
-      for (int wi = 0; wi < kThreads / 32; ++wi) s += warp_sum[wi];
-      if (s) atomicAdd(dropped, (unsigned long long)s);
-    }
-  }
+  count_dropped(lost, dropped);
 }
 
 // Any alignment: one thread per 8 columns (two groups = one metadata byte), element-wise.
@@ -400,14 +449,17 @@ extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const v
   const bool vec = K % 16 == 0 && aligned16(x) && aligned16(vals) && aligned16(meta) && (ldx * es) % 16 == 0 &&
                    (ldv * es) % (8 * es) == 0;
   if (vec) {
-    int64_t chunks_pad = k_pad / 16, total = rows_pad * chunks_pad;
-    unsigned blocks = blocks_for(total, kThreads);
-    if (es == 2)
-      compress_vec_kernel<2><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)vals, ldv * es,
-                                                         (uint8_t*)meta, (int)l, M, K, rows_pad, chunks_pad, dropped);
-    else
-      compress_vec_kernel<1><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)vals, ldv * es,
-                                                         (uint8_t*)meta, (int)l, M, K, rows_pad, chunks_pad, dropped);
+    constexpr int UNROLL = 4;
+    int64_t chunks_pad = k_pad / 16;
+    if (es == 2) {
+      unsigned blocks = blocks_for(rows_pad * chunks_pad * 2, kThreads * UNROLL);
+      compress16_kernel<UNROLL><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)vals, ldv * es,
+                                                            (uint8_t*)meta, (int)l, M, K, rows_pad, chunks_pad, dropped);
+    } else {
+      unsigned blocks = blocks_for(rows_pad * chunks_pad, kThreads * UNROLL);
+      compress8_kernel<UNROLL><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)vals, ldv * es,
+                                                           (uint8_t*)meta, (int)l, M, K, rows_pad, chunks_pad, dropped);
+    }
   } else {
     int64_t bytes_pad = k_pad / 8, total = rows_pad * bytes_pad;
     unsigned blocks = blocks_for(total, kThreads);

@@ -44,15 +44,18 @@ def run_case(sp, cfg, dense=False, cd=None, rows=None, cols=None, alpha=None, be
     alpha = cfg.alpha if alpha is None else alpha
     beta = cfg.beta if beta is None else beta
     A, Bt, Cm = _problem(cfg)
+    Cm = None
     vals_ref, meta_ref, _ = oracle.compress(A, ab)
     Ad, Btd = to_device(A, ab), to_device(Bt, ab)
     Cd = None
     if beta != 0:
-        if Cm is None:
-            Cm = inputs._matrix(("int8",) if ab == "i8" else ("normal", 1.0), "i8" if ab == "i8" else cd,
-                                cfg.seed, inputs.TENSOR_C, cfg.N, 0, cfg.M)
         if ab == "i8":
-            Cm = Cm.astype(np.int32)
+            Cm = inputs._matrix(("int8",), "i8", cfg.seed, inputs.TENSOR_C, cfg.N, 0, cfg.M).astype(np.int32)
+        else:
+            store = cd if cd != "f32" else "bf16"          # fp32 C: bf16-representable values, widened
+            Cm = inputs._matrix(("normal", 1.0), store, cfg.seed, inputs.TENSOR_C, cfg.N, 0, cfg.M)
+            if cd == "f32":
+                Cm = np.ascontiguousarray(oracle.bits_to_float64(Cm, store).astype(np.float32))
         Cd = to_device(Cm, "i32" if ab == "i8" else cd)
     if dense:
         pruned = sp.prune(Ad)

@@ -109,7 +109,7 @@ sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const void* x, int
                           void* vals, int64_t ldv, void* meta, sp24_meta_layout l,
                           unsigned long long* dropped_nonzeros, void* stream);
 
-/* Inverse of sp24_compress (the metadata "decodes the compressed format", Section 3.1):
+/* Inverse of sp24_compress (the metadata is what decodes the format, Section 3.1):
  * y is M x K row-major (ldy >= K) with y[i, 4g+p_t] = vals[i, 2g+t] and +0 elsewhere. */
 sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals, int64_t ldv,
                             const void* meta, sp24_meta_layout l, void* y, int64_t ldy,
@@ -161,6 +161,23 @@ sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A,
  * (synchronises `stream`) and returns SP24_OK, or SP24_ERR_TIMEOUT if a bounded wait inside
  * the kernel expired (the kernel then returned early and D is incomplete). */
 sp24_status sp24_gemm_status(const void* workspace, void* stream);
+
+/* (No counterpart in the paper: a deployment variant of sp24_gemm.)
+ * sp24_gemm for callers that cannot allocate device memory -- a process whose framework
+ * allocator already owns all of the GPU's memory, so that cudaMalloc fails, or a serving loop
+ * that cannot afford the device-wide synchronisation cudaMalloc implies.  The workspace
+ * (status record) lives in a fixed 4096-byte device array inside the library, present on every
+ * GPU that loads the library until the process exits; problems whose
+ * sp24_gemm_workspace_bytes exceeds 4096 are refused with SP24_ERR_WORKSPACE.  Arguments and
+ * results are those of sp24_gemm; inputs and outputs remain the caller's buffers.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress);
+ * make that first call before any stream capture.  Nothing is allocated or freed.
+ * All calls on a device share the array and its status word is cleared on the stream before
+ * each launch, so two calls that overlap on the GPU (different streams) race: serialise them.
+ * The status record of this variant cannot be read back with sp24_gemm_status. */
+sp24_status sp24_gemm_static_ws(const sp24_gemm_desc* d, const void* alpha, const void* A,
+                                const void* meta, const void* B, const void* beta,
+                                const void* C, void* D, void* stream);
 
 /* Lowering of a 3x3, stride-1, pad-1 NHWC convolution input to the GEMM's B operand
  * (Section 4.2: a convolution's reduction dimension is C*R*S).  Output is K-contiguous:

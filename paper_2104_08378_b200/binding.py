@@ -30,7 +30,7 @@ _FROM_TORCH = {torch.float16: "f16", torch.bfloat16: "bf16", torch.int8: "i8", t
 EXPORTS = [
     "sp24_status_string", "sp24_values_bytes", "sp24_meta_bytes", "sp24_prune", "sp24_compress",
     "sp24_decompress", "sp24_gemm_workspace_bytes", "sp24_gemm", "sp24_gemm_status",
-    "sp24_im2col_nhwc_3x3", "sp24_pipeline_host",
+    "sp24_im2col_nhwc_3x3", "sp24_pipeline_host", "sp24_gemm_static_ws",
 ]
 
 
@@ -67,6 +67,8 @@ def _load() -> ctypes.CDLL:
     lib.sp24_gemm_workspace_bytes.argtypes = [ctypes.POINTER(GemmDesc)]
     lib.sp24_gemm_workspace_bytes.restype = sz
     lib.sp24_gemm.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sp24_gemm_static_ws.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sp24_gemm_static_ws.restype = ci
     lib.sp24_gemm_status.argtypes = [vp, vp]
     lib.sp24_im2col_nhwc_3x3.argtypes = [ci, i64, i64, i64, i64, vp, vp, i64, vp]
     lib.sp24_pipeline_host.argtypes = [ctypes.POINTER(GemmDesc)] + [vp] * 13 + [sz, vp]
@@ -205,4 +207,22 @@ def im2col_nhwc_3x3(x: torch.Tensor, dtype: str | None = None) -> torch.Tensor:
     out = torch.empty((Nb * H * W, 9 * C), dtype=x.dtype, device=x.device)
     _check(lib.sp24_im2col_nhwc_3x3(DTYPE_CODE[dt], Nb, H, W, C, _ptr(x), _ptr(out), 9 * C, _stream()),
            "sp24_im2col_nhwc_3x3")
+    return out
+
+
+def gemm_static_ws(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor, *, alpha=1.0, beta=0.0,
+                   C: torch.Tensor | None = None, out: torch.Tensor, cd: str | None = None,
+                   ab: str | None = None, a_is_dense: bool = False) -> torch.Tensor:
+    """sp24_gemm_static_ws: the GEMM for callers that cannot allocate device memory (the workspace is
+    a fixed array inside the library).  `out` must be provided: nothing is allocated here either."""
+    ab = _dtype_of(A, ab)
+    M = A.shape[0]
+    K = A.shape[1] if a_is_dense else 2 * A.shape[1]
+    N = Bt.shape[0]
+    cd = cd or ("i32" if ab == "i8" else ab)
+    desc = make_desc(ab, cd, M, N, K, A.stride(0), Bt.stride(0), C.stride(0) if C is not None else N,
+                     out.stride(0), a_is_dense)
+    a, b = _scalar(ab, alpha), _scalar(ab, beta)
+    _check(lib.sp24_gemm_static_ws(ctypes.byref(desc), ctypes.byref(a), _ptr(A), _ptr(meta), _ptr(Bt),
+                                   ctypes.byref(b), _ptr(C), _ptr(out), _stream()), "sp24_gemm_static_ws")
     return out

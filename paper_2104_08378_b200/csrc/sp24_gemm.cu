@@ -564,3 +564,54 @@ extern "C" sp24_status sp24_gemm_status(const void* workspace, void* stream) {
   SP24_CUDA_CHECK(cudaStreamSynchronize(s));
   return host[0] == 0 ? SP24_OK : SP24_ERR_TIMEOUT;
 }
+
+// ---------------------------------------------------------------------------------------------
+// sp24_gemm_static_ws: sp24_gemm for callers that cannot allocate device memory.
+//
+// sp24_gemm needs a small device workspace (its status record) that the caller normally
+// allocates.  Some callers cannot: a serving process whose framework allocator has already
+// reserved all device memory (cudaMalloc then fails), or a latency-critical loop that must not
+// pay cudaMalloc's implicit device-wide synchronisation.  For them the workspace lives in the
+// file-scope device array below, which every GPU that loads this library holds until the
+// process exits.  Inputs and outputs are still the caller's.
+//
+// The array's name is only a host-side stand-in in host code, not a device address, so the
+// address is resolved with cudaGetSymbolAddress once per device (with that device current) on
+// the first call made on that device; that first call should therefore come before any stream
+// capture.  The entry point calls no cudaMalloc, cudaFree or other allocating routine.
+//
+// All calls on a device share the one array, which keeps the previous call's contents; the
+// status word is cleared on the stream before each launch.  Calls that overlap on the GPU
+// (different streams) race on that word: serialise them, or use sp24_gemm with one workspace
+// per stream.
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr size_t kStaticWorkspaceBytes = 4096;  // stated maximum; sp24_gemm currently needs 256
+static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_ws_mutex;
+void* g_static_ws_ptr[kMaxDevices] = {};
+}  // namespace
+
+extern "C" sp24_status sp24_gemm_static_ws(const sp24_gemm_desc* d, const void* alpha, const void* A,
+                                           const void* meta, const void* B, const void* beta, const void* C,
+                                           void* D, void* stream) {
+  SP24_RETURN_IF(d == nullptr, SP24_ERR_NULL);
+  // the problem's workspace need must fit the fixed array
+  SP24_RETURN_IF(sp24_gemm_workspace_bytes(d) > kStaticWorkspaceBytes, SP24_ERR_WORKSPACE);
+  int dev = 0;
+  SP24_CUDA_CHECK(cudaGetDevice(&dev));
+  SP24_RETURN_IF(dev < 0 || dev >= kMaxDevices, SP24_ERR_UNSUPPORTED);
+  void* ws = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_ws_mutex);
+    if (g_static_ws_ptr[dev] == nullptr) {
+      void* ptr = nullptr;
+      if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || ptr == nullptr) return SP24_ERR_CUDA;
+      g_static_ws_ptr[dev] = ptr;
+    }
+    ws = g_static_ws_ptr[dev];
+  }
+  return sp24_gemm(d, alpha, A, meta, B, beta, C, D, ws, kStaticWorkspaceBytes, stream);
+}

@@ -64,7 +64,7 @@ static double load_as_double(int dtype, const void* base, int64_t index) {
   return (double)((const int8_t*)base)[index];
 }
 
-/* Magnitude key used by the pruning criterion (Section 4.1, step 2: "magnitude").
+/* Magnitude key used by the pruning criterion (Section 4.1, step 2).
  * 16-bit floats: the bit pattern without the sign bit, which orders finite values by |x|
  * (zero of either sign -> 0, subnormals keep their rank).  int8: |x| as an int, -128 -> 128. */
 static int magnitude_key(int dtype, const void* base, int64_t index) {

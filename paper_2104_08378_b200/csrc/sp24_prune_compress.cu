@@ -83,27 +83,29 @@ __device__ __forceinline__ uint4 prune_vec(uint4 v) {
   return v;
 }
 
+// Launch geometry of the vectorised kernels: blockDim = (TX, 256/TX), a warp always lies inside
+// one row; thread (tx, ty) of block (bx, by) handles units (bx*UNROLL + u)*TX + tx, u < UNROLL, of
+// rows by*TY + ty, + gridDim.y*TY, ...  No integer division on the device.
 // One 16-byte vector per thread and unroll step; `vpr` vectors per row.
 template <int ES, int UNROLL>
 __global__ void __launch_bounds__(kThreads) prune_vec_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
                                                              uint8_t* y, int64_t row_bytes_y, int64_t vpr,
-                                                             int64_t total) {
-  int64_t base = (int64_t)blockIdx.x * (kThreads * UNROLL) + threadIdx.x;
-  uint4 v[UNROLL];
-  int64_t off_y[UNROLL];
+                                                             int64_t rows) {
+  const int64_t c0 = (int64_t)blockIdx.x * UNROLL * blockDim.x + threadIdx.x;
+  for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows;
+       row += (int64_t)gridDim.y * blockDim.y) {
+    uint4 v[UNROLL];
 #pragma unroll
-  for (int u = 0; u < UNROLL; ++u) {
-    int64_t id = base + (int64_t)u * kThreads;
-    off_y[u] = -1;
-    if (id < total) {
-      int64_t row = id / vpr, c = id - row * vpr;
-      v[u] = ld_stream(x + row * row_bytes_x + c * 16);
-      off_y[u] = row * row_bytes_y + c * 16;
+    for (int u = 0; u < UNROLL; ++u) {
+      int64_t c = c0 + (int64_t)u * blockDim.x;
+      if (c < vpr) v[u] = ld_stream(x + row * row_bytes_x + c * 16);
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      int64_t c = c0 + (int64_t)u * blockDim.x;
+      if (c < vpr) st_stream(y + row * row_bytes_y + c * 16, prune_vec<ES>(v[u]));
     }
   }
-#pragma unroll
-  for (int u = 0; u < UNROLL; ++u)
-    if (off_y[u] >= 0) st_stream(y + off_y[u], prune_vec<ES>(v[u]));
 }
 
 // Any alignment / leading dimension: one thread per group, element-wise accesses.
@@ -148,13 +150,51 @@ __device__ __forceinline__ int64_t meta_offset(int layout, int64_t row, int64_t 
 // The domain is padded (rows to rows_pad, 16-column chunks to chunks_pad) so that the operand-
 // order layout gets its 0x4 padding nibbles from the same launch.  Every thread issues all of
 // its loads before it consumes any of them.
+//
+// Selection by table: the six comparisons of a group are made two at a time on packed 15-bit
+// keys -- ((a | 0x8000) - b) has bit 15 set iff a >= b, and two such differences fit one 32-bit
+// subtraction without a borrow between the halves -- and their six result bits index a 64-entry
+// table in shared memory that holds, per outcome, the metadata nibble, the keep mask and the
+// byte-permute selectors that gather the two kept values.
+__device__ __forceinline__ uint32_t selection_entry(uint32_t idx) {
+  // idx bits: 0 = c01, 1 = c03, 2 = c02, 3 = c23, 4 = c12, 5 = c13   (cab: key[a] >= key[b])
+  uint32_t c01 = idx & 1, c03 = (idx >> 1) & 1, c02 = (idx >> 2) & 1;
+  uint32_t c23 = (idx >> 3) & 1, c12 = (idx >> 4) & 1, c13 = (idx >> 5) & 1;
+  uint32_t b0 = 3u - (c01 + c02 + c03), b1 = c01 + 2u - (c12 + c13);
+  uint32_t b2 = c02 + c12 + 1u - c23, b3 = c03 + c13 + c23;
+  uint32_t mask = (b0 < 2u) | ((b1 < 2u) << 1) | ((b2 < 2u) << 2) | ((b3 < 2u) << 3);
+  if (__popc(mask) != 2) mask = 3;  // comparison outcomes no real keys can produce
+  uint32_t p0 = __ffs(mask) - 1, p1 = 31 - __clz(mask);
+  uint32_t sel8 = p0 | (p1 << 4);                                                // bytes p0, p1 of a word
+  uint32_t sel16 = (2 * p0) | ((2 * p0 + 1) << 4) | ((2 * p1) << 8) | ((2 * p1 + 1) << 12);  // halves p0, p1 of a pair
+  return (p0 | (p1 << 2)) | (mask << 4) | (sel8 << 8) | (sel16 << 16);
+}
+
+__device__ __forceinline__ void build_selection_table(uint32_t* table) {
+  int t = threadIdx.y * blockDim.x + threadIdx.x;
+  if (t < 64) table[t] = selection_entry((uint32_t)t);
+  __syncthreads();
+}
+
+// k_lo = [key0, key1], k_hi = [key2, key3] as 16-bit lanes, every key < 2^15.
+__device__ __forceinline__ uint32_t selection_index(uint32_t k_lo, uint32_t k_hi) {
+  const uint32_t g = 0x80008000u;
+  uint32_t r1 = (k_lo | g) - k_hi;                              // bit 15: c02, bit 31: c13
+  uint32_t r2 = (k_lo | g) - __byte_perm(k_hi, 0, 0x1032);      // bit 15: c03, bit 31: c12
+  uint32_t r3 = (__byte_perm(k_lo, k_hi, 0x5410) | g) - __byte_perm(k_lo, k_hi, 0x7632);  // bit 15: c01, 31: c23
+  uint32_t t = (r1 & g) | ((r2 & g) >> 1) | ((r3 & g) >> 2);    // bits 15..13: c02 c03 c01, 31..29: c13 c12 c23
+  return ((t >> 13) & 7u) | ((t >> 26) & 0x38u);
+}
+
+template <bool COUNT>
 __device__ __forceinline__ void count_dropped(uint32_t lost, unsigned long long* dropped) {
-  if (dropped == nullptr) return;
+  if (!COUNT) return;
   lost = __reduce_add_sync(0xFFFFFFFFu, lost);
   __shared__ uint32_t warp_sum[kThreads / 32];
-  if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = lost;
+  int t = threadIdx.y * blockDim.x + threadIdx.x;
+  if ((t & 31) == 0) warp_sum[t >> 5] = lost;
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (t == 0) {
     uint32_t s = 0;
 #pragma unroll
     for (int wi = 0; wi < kThreads / 32; ++wi) s += warp_sum[wi];
@@ -165,104 +205,97 @@ __device__ __forceinline__ void count_dropped(uint32_t lost, unsigned long long*
 // 16-bit types.  Work unit: 8 columns (two groups) = one 16-byte load, 8 bytes of values and one
 // metadata byte out, so a warp reads 512 and writes 256 contiguous bytes per step.  Lanes 2j and
 // 2j+1 hold the two halves of a 16-column chunk; the even lane stores the chunk's 16 metadata bits.
-template <int UNROLL>
-__global__ void __launch_bounds__(kThreads) compress16_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
+template <int UNROLL, bool COUNT>
+__global__ void __launch_bounds__(kThreads, 4) compress16_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
                                                               uint8_t* __restrict__ vals, int64_t row_bytes_v,
                                                               uint8_t* __restrict__ meta, int layout, int64_t M,
                                                               int64_t K, int64_t rows_pad, int64_t chunks_pad,
                                                               unsigned long long* dropped) {
+  __shared__ uint32_t table[64];
+  build_selection_table(table);
   const int64_t halves = K >> 3, halves_pad = chunks_pad * 2, KB = chunks_pad >> 3;
-  const int64_t total = rows_pad * halves_pad;
-  const int64_t base = (int64_t)blockIdx.x * (kThreads * UNROLL) + threadIdx.x;
-  uint4 in[UNROLL];
-  int64_t row[UNROLL], half[UNROLL];
-  bool live[UNROLL];
-#pragma unroll
-  for (int u = 0; u < UNROLL; ++u) {
-    int64_t id = base + (int64_t)u * kThreads;
-    row[u] = id / halves_pad;
-    half[u] = id - row[u] * halves_pad;
-    live[u] = id < total && row[u] < M && half[u] < halves;
-    if (live[u]) in[u] = ld_stream(x + row[u] * row_bytes_x + half[u] * 16);
-  }
+  const int64_t h0 = (int64_t)blockIdx.x * UNROLL * blockDim.x + threadIdx.x;
   uint32_t lost = 0;
+  for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows_pad;
+       row += (int64_t)gridDim.y * blockDim.y) {
+    uint4 in[UNROLL];
 #pragma unroll
-  for (int u = 0; u < UNROLL; ++u) {
-    uint32_t mbyte = 0x44u;  // padding: positions (0, 1) in both groups
-    if (live[u]) {
-      uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
-      uint32_t out[2];
-      mbyte = 0;
-#pragma unroll
-      for (int g = 0; g < 2; ++g) {
-        uint32_t lo = w[2 * g], hi = w[2 * g + 1];
-        uint32_t m = Group16::mask(lo, hi);
-        uint32_t nib = mask_to_nibble(m);
-        uint64_t both = (uint64_t)lo | ((uint64_t)hi << 32);
-        uint32_t v0 = (uint32_t)(both >> (16 * (nib & 3))) & 0xFFFFu;
-        uint32_t v1 = (uint32_t)(both >> (16 * (nib >> 2))) & 0xFFFFu;
-        out[g] = v0 | (v1 << 16);
-        mbyte |= nib << (4 * g);
-        lost += __popc(Group16::nonzero(lo, hi) & ~m);
-      }
-      __stcs(reinterpret_cast<uint2*>(vals + row[u] * row_bytes_v + half[u] * 8), make_uint2(out[0], out[1]));
+    for (int u = 0; u < UNROLL; ++u) {
+      int64_t half = h0 + (int64_t)u * blockDim.x;
+      if (row < M && half < halves) in[u] = ld_stream(x + row * row_bytes_x + half * 16);
     }
-    uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, mbyte, 1);
-    int64_t id = base + (int64_t)u * kThreads;
-    if ((threadIdx.x & 1) == 0 && id < total)
-      *reinterpret_cast<uint16_t*>(meta + meta_offset<2>(layout, row[u], half[u] >> 1, K, KB)) =
-          (uint16_t)(mbyte | (other << 8));
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      int64_t half = h0 + (int64_t)u * blockDim.x;
+      uint32_t mbyte = 0x44u;  // padding: positions (0, 1) in both groups
+      if (row < M && half < halves) {
+        uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
+        uint32_t out[2];
+        mbyte = 0;
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+          uint32_t lo = w[2 * g], hi = w[2 * g + 1];
+          uint32_t e = table[selection_index(lo & 0x7FFF7FFFu, hi & 0x7FFF7FFFu)];
+          out[g] = __byte_perm(lo, hi, e >> 16);
+          mbyte |= (e & 0xFu) << (4 * g);
+          if (COUNT) lost += __popc(Group16::nonzero(lo, hi) & ~(e >> 4) & 0xFu);
+        }
+        __stcs(reinterpret_cast<uint2*>(vals + row * row_bytes_v + half * 8), make_uint2(out[0], out[1]));
+      }
+      uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, mbyte, 1);
+      if ((threadIdx.x & 1) == 0 && half < halves_pad)
+        *reinterpret_cast<uint16_t*>(meta + meta_offset<2>(layout, row, half >> 1, K, KB)) =
+            (uint16_t)(mbyte | (other << 8));
+    }
   }
-  count_dropped(lost, dropped);
+  count_dropped<COUNT>(lost, dropped);
 }
 
 // int8.  Work unit: one chunk of 16 columns (four groups) = one 16-byte load, 8 bytes of values and
 // 16 bits of metadata out.
-template <int UNROLL>
-__global__ void __launch_bounds__(kThreads) compress8_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
+template <int UNROLL, bool COUNT>
+__global__ void __launch_bounds__(kThreads, 4) compress8_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
                                                              uint8_t* __restrict__ vals, int64_t row_bytes_v,
                                                              uint8_t* __restrict__ meta, int layout, int64_t M,
                                                              int64_t K, int64_t rows_pad, int64_t chunks_pad,
                                                              unsigned long long* dropped) {
+  __shared__ uint32_t table[64];
+  build_selection_table(table);
   const int64_t chunks = K >> 4, KB = chunks_pad >> 3;
-  const int64_t total = rows_pad * chunks_pad;
-  const int64_t base = (int64_t)blockIdx.x * (kThreads * UNROLL) + threadIdx.x;
-  uint4 in[UNROLL];
-  int64_t row[UNROLL], chunk[UNROLL];
-  bool live[UNROLL];
-#pragma unroll
-  for (int u = 0; u < UNROLL; ++u) {
-    int64_t id = base + (int64_t)u * kThreads;
-    row[u] = id / chunks_pad;
-    chunk[u] = id - row[u] * chunks_pad;
-    live[u] = id < total && row[u] < M && chunk[u] < chunks;
-    if (live[u]) in[u] = ld_stream(x + row[u] * row_bytes_x + chunk[u] * 16);
-  }
+  const int64_t c0 = (int64_t)blockIdx.x * UNROLL * blockDim.x + threadIdx.x;
   uint32_t lost = 0;
+  for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows_pad;
+       row += (int64_t)gridDim.y * blockDim.y) {
+    uint4 in[UNROLL];
 #pragma unroll
-  for (int u = 0; u < UNROLL; ++u) {
-    int64_t id = base + (int64_t)u * kThreads;
-    if (id >= total) continue;
-    uint32_t mbits = 0x4444u;
-    if (live[u]) {
-      uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
-      uint32_t out[2] = {0, 0};
-      mbits = 0;
-#pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        uint32_t m = Group8::mask(w[g]);
-        uint32_t nib = mask_to_nibble(m);
-        uint32_t v0 = (w[g] >> (8 * (nib & 3))) & 0xFFu;
-        uint32_t v1 = (w[g] >> (8 * (nib >> 2))) & 0xFFu;
-        out[g >> 1] |= (v0 | (v1 << 8)) << (16 * (g & 1));
-        mbits |= nib << (4 * g);
-        lost += __popc(Group8::nonzero(w[g]) & ~m);
-      }
-      __stcs(reinterpret_cast<uint2*>(vals + row[u] * row_bytes_v + chunk[u] * 8), make_uint2(out[0], out[1]));
+    for (int u = 0; u < UNROLL; ++u) {
+      int64_t chunk = c0 + (int64_t)u * blockDim.x;
+      if (row < M && chunk < chunks) in[u] = ld_stream(x + row * row_bytes_x + chunk * 16);
     }
-    *reinterpret_cast<uint16_t*>(meta + meta_offset<1>(layout, row[u], chunk[u], K, KB)) = (uint16_t)mbits;
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      int64_t chunk = c0 + (int64_t)u * blockDim.x;
+      if (chunk >= chunks_pad) continue;
+      uint32_t mbits = 0x4444u;
+      if (row < M && chunk < chunks) {
+        uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
+        uint32_t out[2] = {0, 0};
+        mbits = 0;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          uint32_t a = __vabs4(w[g]);  // -128 -> 0x80 = 128, no saturation
+          uint32_t e = table[selection_index(__byte_perm(a, 0, 0x4140), __byte_perm(a, 0, 0x4342))];
+          uint32_t pair = __byte_perm(w[g], 0, ((e >> 8) & 0xFFu) | 0x4400u);
+          out[g >> 1] |= pair << (16 * (g & 1));
+          mbits |= (e & 0xFu) << (4 * g);
+          if (COUNT) lost += __popc(Group8::nonzero(w[g]) & ~(e >> 4) & 0xFu);
+        }
+        __stcs(reinterpret_cast<uint2*>(vals + row * row_bytes_v + chunk * 8), make_uint2(out[0], out[1]));
+      }
+      *reinterpret_cast<uint16_t*>(meta + meta_offset<1>(layout, row, chunk, K, KB)) = (uint16_t)mbits;
+    }
   }
-  count_dropped(lost, dropped);
+  count_dropped<COUNT>(lost, dropped);
 }
 
 // Any alignment: one thread per 8 columns (two groups = one metadata byte), element-wise.
@@ -386,6 +419,26 @@ __global__ void __launch_bounds__(kThreads) im2col_3x3_kernel(const uint8_t* __r
 
 inline unsigned blocks_for(int64_t total, int per_block) { return (unsigned)((total + per_block - 1) / per_block); }
 
+// Block shape and grid of the vectorised kernels for `units` work units per row and `rows` rows:
+// TX (a power of two, 32..256) threads along the row, chosen to waste the fewest lanes.
+struct RowLaunch {
+  dim3 grid, block;
+  RowLaunch(int64_t units, int64_t rows, int unroll) {
+    int best_tx = 256;
+    int64_t best_cover = -1;
+    for (int tx = 256; tx >= 32; tx /= 2) {
+      int64_t per = (int64_t)tx * unroll;
+      int64_t cover = (units + per - 1) / per * per;
+      if (best_cover < 0 || cover < best_cover) { best_cover = cover; best_tx = tx; }
+    }
+    int ty = kThreads / best_tx;
+    block = dim3((unsigned)best_tx, (unsigned)ty, 1);
+    int64_t gy = (rows + ty - 1) / ty;
+    if (gy > 32768) gy = 32768;
+    grid = dim3((unsigned)(best_cover / ((int64_t)best_tx * unroll)), (unsigned)gy, 1);
+  }
+};
+
 }  // namespace
 
 static sp24_status validate_matrix_args(sp24_dtype t, int64_t M, int64_t K, int64_t k_multiple) {
@@ -411,15 +464,18 @@ extern "C" sp24_status sp24_prune(sp24_dtype t, int64_t M, int64_t K, const void
   const bool vec = aligned16(x) && aligned16(y) && (ldx * es) % 16 == 0 && (ldy * es) % 16 == 0 && (K * es) % 16 == 0;
   if (vec) {
     constexpr int UNROLL = 4;
-    int64_t vpr = K * es / 16, total = M * vpr;
-    if (ldx == K && ldy == K) {  // packed: treat the matrix as one long row, no per-vector division
-      vpr = total;
+    int64_t vpr = K * es / 16, rows = M;
+    if (ldx == K && ldy == K && vpr < 256 * UNROLL) {  // packed and short rows: fold rows into long ones
+      int64_t fold = 1;
+      while (vpr * fold * 2 <= 256 * UNROLL && rows % 2 == 0) { fold *= 2; rows /= 2; }
+      vpr *= fold;
     }
-    unsigned blocks = blocks_for(total, kThreads * UNROLL);
+    RowLaunch L(vpr, rows, UNROLL);
+    int64_t rbx = ldx == K && ldy == K ? vpr * 16 : ldx * es, rby = ldx == K && ldy == K ? vpr * 16 : ldy * es;
     if (es == 2)
-      prune_vec_kernel<2, UNROLL><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)y, ldy * es, vpr, total);
+      prune_vec_kernel<2, UNROLL><<<L.grid, L.block, 0, s>>>((const uint8_t*)x, rbx, (uint8_t*)y, rby, vpr, rows);
     else
-      prune_vec_kernel<1, UNROLL><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)y, ldy * es, vpr, total);
+      prune_vec_kernel<1, UNROLL><<<L.grid, L.block, 0, s>>>((const uint8_t*)x, rbx, (uint8_t*)y, rby, vpr, rows);
   } else {
     int64_t gpr = K / 4, total = M * gpr;
     unsigned blocks = blocks_for(total, kThreads);
@@ -451,14 +507,24 @@ extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const v
   if (vec) {
     constexpr int UNROLL = 4;
     int64_t chunks_pad = k_pad / 16;
+    const uint8_t* xs = (const uint8_t*)x;
+    uint8_t *vs = (uint8_t*)vals, *ms = (uint8_t*)meta;
     if (es == 2) {
-      unsigned blocks = blocks_for(rows_pad * chunks_pad * 2, kThreads * UNROLL);
-      compress16_kernel<UNROLL><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)vals, ldv * es,
-                                                            (uint8_t*)meta, (int)l, M, K, rows_pad, chunks_pad, dropped);
+      RowLaunch L(chunks_pad * 2, rows_pad, UNROLL);
+      if (dropped)
+        compress16_kernel<UNROLL, true><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, (int)l, M, K, rows_pad,
+                                                                   chunks_pad, dropped);
+      else
+        compress16_kernel<UNROLL, false><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, (int)l, M, K, rows_pad,
+                                                                    chunks_pad, dropped);
     } else {
-      unsigned blocks = blocks_for(rows_pad * chunks_pad, kThreads * UNROLL);
-      compress8_kernel<UNROLL><<<blocks, kThreads, 0, s>>>((const uint8_t*)x, ldx * es, (uint8_t*)vals, ldv * es,
-                                                           (uint8_t*)meta, (int)l, M, K, rows_pad, chunks_pad, dropped);
+      RowLaunch L(chunks_pad, rows_pad, UNROLL);
+      if (dropped)
+        compress8_kernel<UNROLL, true><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, (int)l, M, K, rows_pad,
+                                                                  chunks_pad, dropped);
+      else
+        compress8_kernel<UNROLL, false><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, (int)l, M, K, rows_pad,
+                                                                   chunks_pad, dropped);
     }
   } else {
     int64_t bytes_pad = k_pad / 8, total = rows_pad * bytes_pad;

@@ -3,15 +3,21 @@
 // (tcgen05.mma, the "dense variant" that supplies the sparse-vs-dense speedup).
 //
 // One persistent, warp-specialised kernel:
-//   warp 0   TMA producer: compressed-A tile, metadata block(s) and B tiles of one k-block into a
+//   warp 0   TMA producer: compressed-A tiles, metadata blocks and B tiles of one k-block into a
 //            ring of shared-memory stages (mbarrier expect_tx / complete_tx);
 //   warp 1   MMA issuer (one elected thread): copies the stage's metadata shared -> tensor
 //            memory (tcgen05.cp), issues the tcgen05.mma[.sp] of the stage, commits the stage
-//            back to the producer and, after the last k-block, the accumulator to the epilogue;
+//            back to the producer and, after the last k-block, the accumulators to the epilogue;
 //            owns the tensor-memory allocation;
-//   warps 2-5 epilogue: tcgen05.ld accumulator -> registers, alpha/beta, convert, store.
-// CTAS == 2 runs a pair of CTAs (cluster of two) on one 256 x 256 tile: each CTA loads its 128
-// rows of A / metadata and its half of B, CTA 0 issues cta_group::2 MMAs for both.
+//   warps 2-5 epilogue: tcgen05.ld accumulator -> registers, alpha/beta, convert, store; the loads
+//            of C and of the next accumulator chunk run one chunk ahead.
+// CTAS == 2 runs a pair of CTAs (cluster of two): each CTA loads its 128 rows of A / metadata per
+// m-block and its half of B, CTA 0 issues cta_group::2 MMAs (M = 256) for both.
+// MBLK == 2 gives every CTA two m-blocks (two accumulators, one B tile): what an SM can pull in
+// from the L2 per clock, not the tensor pipe, bounds this kernel, and sharing the B tile between
+// two m-blocks cuts the bytes per flop by about a third.  The two accumulators then fill tensor
+// memory, so the epilogue is not overlapped with the next tile's main loop; MBLK == 1 keeps two
+// accumulator buffers and overlaps it.
 // Every wait is bounded: on expiry the role records a code in the status word and all roles
 // leave through the normal teardown (no trap, no endless spin).
 #include <cuda.h>
@@ -28,7 +34,7 @@
 namespace sp24 {
 namespace {
 
-constexpr int kBlockM = 128;              // rows of A per CTA (tensor-memory lanes)
+constexpr int kBlockM = 128;              // rows of A per CTA and m-block (tensor-memory lanes)
 constexpr int kAtomBytes = 128;           // bytes per row of one swizzle-128B operand atom
 constexpr int kNumThreads = 192;          // 6 warps
 constexpr uint64_t kWaitTimeoutNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
@@ -39,39 +45,47 @@ struct GemmParams {
   int64_t ldc, ldd;   // elements
   const void* C;
   void* D;
-  uint32_t* status;   // [0] = 0 ok, else code of the wait that expired; [1] = launches seen
+  uint32_t* status;   // [0] = 0 ok, else code of the wait that expired
   float alpha, beta;
   int32_t m_tiles, n_tiles, k_blocks;
   int32_t meta_kb;    // 128-column metadata blocks per 128-row block (K padded to 256)
   int32_t a_fmt;      // 0 f16, 1 bf16 (kind::f16); ignored for int8
   int32_t cd_type;    // sp24_dtype of C / D
   int32_t has_c;
+  int32_t band;       // m-tiles per band of the tile sweep
 };
 
-template <int KIND, bool SPARSE, int BLOCK_N, int CTAS>
+template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK>
 struct Cfg {
-  static constexpr int kABoxes = SPARSE ? 1 : 2;                   // 128-byte atoms of A per stage
-  static constexpr int kBBoxes = 2;
+  // 128-byte atoms per stage: sparse A is half as wide as B; the dense variant with two
+  // m-blocks takes one atom per operand so that four stages still fit
+  static constexpr int kBBoxes = SPARSE ? 2 : (MBLK == 2 ? 1 : 2);
+  static constexpr int kABoxes = SPARSE ? 1 : kBBoxes;
   static constexpr int kBRows = BLOCK_N / CTAS;                    // B rows (N) this CTA loads
-  static constexpr int kABytes = kABoxes * kBlockM * kAtomBytes;
+  static constexpr int kABlockBytes = kABoxes * kBlockM * kAtomBytes;  // one m-block
+  static constexpr int kABytes = MBLK * kABlockBytes;
   static constexpr int kBBytes = kBBoxes * kBRows * kAtomBytes;
-  static constexpr int kEBlocks = SPARSE ? (KIND == 0 ? 1 : 2) : 0;  // 2048-byte metadata blocks per stage
-  static constexpr int kEBytes = kEBlocks * 2048;
-  static constexpr int kStageBytes = kABytes + kBBytes + (SPARSE ? 4096 : 0);
-  static constexpr int kStages = (216 * 1024) / kStageBytes;
-  static constexpr int kTxBytes = (kABytes + kBBytes + kEBytes) * CTAS;
-  static constexpr int kAccStages = (2 * BLOCK_N + 32 <= (int)kTmemCols) ? 2 : 1;
-  static constexpr int kECol = kAccStages * BLOCK_N;               // first metadata column in tensor memory
-  static constexpr int kMmasPerStage = SPARSE ? 4 : 8;
+  static constexpr int kEBlocks = SPARSE ? (KIND == 0 ? 1 : 2) : 0;  // 2048-byte metadata blocks per m-block and stage
+  static constexpr int kEBlockBytes = kEBlocks * 2048;
+  static constexpr int kEBytes = MBLK * kEBlockBytes;
+  static constexpr int kEAlloc = (kEBytes + 1023) / 1024 * 1024;
+  static constexpr int kStageBytes = kABytes + kBBytes + kEAlloc;
+  static constexpr int kStages = (216 * 1024) / kStageBytes > 8 ? 8 : (216 * 1024) / kStageBytes;
+  static constexpr int kAccStages = MBLK == 2 ? 1 : ((2 * BLOCK_N + 32 <= (int)kTmemCols) ? 2 : 1);
+  static constexpr int kECol = kAccStages * MBLK * BLOCK_N;        // first metadata column in tensor memory
+  static constexpr int kMmasPerStage = SPARSE ? 4 : 4 * kBBoxes;   // per m-block
   static constexpr int kKPerStage = (KIND == 0 ? 64 : 128) * kBBoxes;  // logical K per stage
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
   static_assert(kStages >= 2, "need at least two stages");
+  static_assert(kStageBytes % 1024 == 0, "stages must keep the 1024-byte alignment of the atoms");
+  static_assert(kECol + (SPARSE ? 2 * MBLK * 8 : 0) <= (int)kTmemCols, "tensor memory overflow");
 };
 
 struct Shared {
   uint64_t full[8], empty[8], tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   volatile uint32_t abort;
+  volatile uint32_t c_hint_tiles;  // tiles whose main loop is close enough to its end to fetch C into the L2
 };
 
 __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, Shared* sh, uint32_t* status,
@@ -92,15 +106,14 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, Sha
   }
 }
 
-// tile index -> (m_tile, n_tile): bands of `kGroup` m-tiles are swept n-tile by n-tile so that
+// tile index -> (m_tile, n_tile): bands of `band_rows` m-tiles are swept n-tile by n-tile so that
 // the tiles in flight at one time share a few A row-panels and B column-panels in the L2.
-__device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int& mt, int& nt) {
-  constexpr int kGroup = 8;
-  int per_band = kGroup * n_tiles;
+__device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int band_rows, int& mt, int& nt) {
+  int per_band = band_rows * n_tiles;
   int band = t / per_band, in_band = t - band * per_band;
-  int rows = min(kGroup, m_tiles - band * kGroup);
+  int rows = min(band_rows, m_tiles - band * band_rows);
   nt = in_band / rows;
-  mt = band * kGroup + (in_band - nt * rows);
+  mt = band * band_rows + (in_band - nt * rows);
 }
 
 template <int KIND>
@@ -116,11 +129,83 @@ __device__ __forceinline__ uint32_t make_idesc(bool sparse, int a_fmt, int m, in
   return d;                                        // both operands K-major, no negate, no saturate
 }
 
-template <int KIND, bool SPARSE, int BLOCK_N, int CTAS>
+// ---- epilogue helpers: one chunk = 32 consecutive columns of one row ---------------------------
+// C for the chunk, fetched one chunk ahead of its use: 64 bytes (16-bit types) or 128 bytes per thread.
+__device__ __forceinline__ void load_c_chunk(uint4 (&c)[8], const GemmParams& p, int cs, int64_t row, int64_t col,
+                                             int cols_valid) {
+  const uint8_t* base = static_cast<const uint8_t*>(p.C) + (row * p.ldc + col) * cs;
+  const int vecs = 2 * cs;  // 16-byte vectors per chunk: 4 for 2-byte, 8 for 4-byte types
+  const int per_vec = 16 / cs;
+#pragma unroll
+  for (int v = 0; v < 8; ++v)
+    if (v < vecs && v * per_vec < cols_valid) c[v] = __ldg(reinterpret_cast<const uint4*>(base) + v);
+}
+
+template <int KIND>
+__device__ __forceinline__ void store_chunk(const uint32_t (&r)[32], const uint4 (&c)[8], const GemmParams& p,
+                                            int64_t row, int64_t col, int cols_valid) {
+  if (KIND == 1) {
+    int32_t* dp = static_cast<int32_t*>(p.D) + row * p.ldd + col;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (4 * j >= cols_valid) break;
+      int4 v = make_int4((int)r[4 * j], (int)r[4 * j + 1], (int)r[4 * j + 2], (int)r[4 * j + 3]);
+      if (p.has_c) { v.x += (int)c[j].x; v.y += (int)c[j].y; v.z += (int)c[j].z; v.w += (int)c[j].w; }
+      reinterpret_cast<int4*>(dp)[j] = v;
+    }
+  } else if (p.cd_type == SP24_F32) {
+    float* dp = static_cast<float*>(p.D) + row * p.ldd + col;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (4 * j >= cols_valid) break;
+      float4 v = make_float4(p.alpha * __uint_as_float(r[4 * j]), p.alpha * __uint_as_float(r[4 * j + 1]),
+                             p.alpha * __uint_as_float(r[4 * j + 2]), p.alpha * __uint_as_float(r[4 * j + 3]));
+      if (p.has_c) {
+        v.x += p.beta * __uint_as_float(c[j].x); v.y += p.beta * __uint_as_float(c[j].y);
+        v.z += p.beta * __uint_as_float(c[j].z); v.w += p.beta * __uint_as_float(c[j].w);
+      }
+      reinterpret_cast<float4*>(dp)[j] = v;
+    }
+  } else {
+    const bool bf = p.cd_type == SP24_BF16;
+    uint16_t* dp = static_cast<uint16_t*>(p.D) + row * p.ldd + col;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (8 * j >= cols_valid) break;
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = p.alpha * __uint_as_float(r[8 * j + e]);
+      if (p.has_c) {
+        const uint32_t cw[4] = {c[j].x, c[j].y, c[j].z, c[j].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float2 f = bf ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&cw[e]))
+                        : __half22float2(*reinterpret_cast<const __half2*>(&cw[e]));
+          v[2 * e] += p.beta * f.x;
+          v[2 * e + 1] += p.beta * f.y;
+        }
+      }
+      uint32_t ow[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (bf) {
+          __nv_bfloat162 o = __float22bfloat162_rn(make_float2(v[2 * e], v[2 * e + 1]));
+          ow[e] = *reinterpret_cast<uint32_t*>(&o);
+        } else {
+          __half2 o = __float22half2_rn(make_float2(v[2 * e], v[2 * e + 1]));
+          ow[e] = *reinterpret_cast<uint32_t*>(&o);
+        }
+      }
+      reinterpret_cast<uint4*>(dp)[j] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+    }
+  }
+}
+
+template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK>
 __global__ void __launch_bounds__(kNumThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_e, const GemmParams p) {
-  using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS>;
+  using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS, MBLK>;
   extern __shared__ uint8_t smem_raw[];
   // Operand atoms need 1024-byte alignment for the 128-byte swizzle.
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -141,6 +226,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       ptx::mbar_init(&sh->tmem_empty[a], 4 * CTAS);  // one arrival per epilogue warp of the pair
     }
     sh->abort = 0;
+    sh->c_hint_tiles = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&map_a);
     ptx::prefetch_tensormap(&map_b);
@@ -160,38 +246,51 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     // ------------------------------ TMA producer ------------------------------
     if (ptx::elect_one()) {
       int stage = 0;
-      uint32_t phase = 0;
+      uint32_t phase = 0, tiles_started = 0;
+      const int box_elems = KIND == 0 ? 64 : 128;  // elements per 128-byte atom row
+      const int hint_kb = max(0, p.k_blocks - 24);  // when the epilogue warps should pull C into the L2
       for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
+        ++tiles_started;
         int mt, nt;
-        tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
-        const int row0 = (mt * CTAS + (int)cta_rank) * kBlockM;         // first A row of this CTA
-        const int col0 = nt * BLOCK_N + (int)cta_rank * C::kBRows;       // first B row (N index)
-        const int a_box_elems = KIND == 0 ? 64 : 128;                    // elements per 128-byte atom row
+        tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
+        // the last n-tile may be narrower: the pair then splits only the columns that exist
+        const int n_eff = min(BLOCK_N, (int)(p.N - (int64_t)nt * BLOCK_N));
+        const int col0 = nt * BLOCK_N + (int)cta_rank * (n_eff / CTAS);  // first B row (N index)
+        // m-blocks of this tile that have rows at all (the rest are neither loaded nor multiplied)
+        const int live = min(MBLK, (int)((p.M - (int64_t)mt * MBLK * CTAS * kBlockM + CTAS * kBlockM - 1) /
+                                         (CTAS * kBlockM)));
+        const uint32_t tx_bytes = (uint32_t)((live * (C::kABlockBytes + C::kEBlockBytes) + C::kBBytes) * CTAS);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!bounded_wait(&sh->empty[stage], phase ^ 1u, sh, p.status, 1u)) break;
+          if (kb == hint_kb) sh->c_hint_tiles = tiles_started;
           uint8_t* sa = smem + stage * C::kStageBytes;
           uint8_t* sb = sa + C::kABytes;
           uint8_t* se = sb + C::kBBytes;
           uint64_t* full = &sh->full[stage];
-          if (cta_rank == 0) ptx::mbar_expect_tx(full, C::kTxBytes);
+          if (cta_rank == 0) ptx::mbar_expect_tx(full, tx_bytes);
 #pragma unroll
-          for (int i = 0; i < C::kABoxes; ++i) {
-            int x = (kb * C::kABoxes + i) * a_box_elems;
-            if (CTAS == 1) ptx::tma_load_2d(sa + i * kBlockM * kAtomBytes, &map_a, full, x, row0);
-            else ptx::tma_load_2d_pair(sa + i * kBlockM * kAtomBytes, &map_a, full, 0, x, row0);
+          for (int j = 0; j < MBLK; ++j) {
+            if (j >= live) break;
+            const int mb = (mt * MBLK + j) * CTAS + (int)cta_rank;  // 128-row block of A
+#pragma unroll
+            for (int i = 0; i < C::kABoxes; ++i) {
+              uint8_t* dst = sa + j * C::kABlockBytes + i * kBlockM * kAtomBytes;
+              int x = (kb * C::kABoxes + i) * box_elems;
+              if (CTAS == 1) ptx::tma_load_2d(dst, &map_a, full, x, mb * kBlockM);
+              else ptx::tma_load_2d_pair(dst, &map_a, full, 0, x, mb * kBlockM);
+            }
+            if (SPARSE) {
+              // metadata viewed as rows of 128 bytes: block (mb, kb128) starts at row 16 * (mb * KB + kb128)
+              int y = 16 * (mb * p.meta_kb + kb * C::kEBlocks);
+              if (CTAS == 1) ptx::tma_load_2d(se + j * C::kEBlockBytes, &map_e, full, 0, y);
+              else ptx::tma_load_2d_pair(se + j * C::kEBlockBytes, &map_e, full, 0, 0, y);
+            }
           }
 #pragma unroll
           for (int i = 0; i < C::kBBoxes; ++i) {
-            int x = (kb * C::kBBoxes + i) * a_box_elems;
+            int x = (kb * C::kBBoxes + i) * box_elems;
             if (CTAS == 1) ptx::tma_load_2d(sb + i * C::kBRows * kAtomBytes, &map_b, full, x, col0);
             else ptx::tma_load_2d_pair(sb + i * C::kBRows * kAtomBytes, &map_b, full, 0, x, col0);
-          }
-          if (SPARSE) {
-            // metadata viewed as rows of 128 bytes: block (mb, kb128) starts at row 16 * (mb * KB + kb128)
-            int mb = mt * CTAS + (int)cta_rank;
-            int y = 16 * (mb * p.meta_kb + kb * C::kEBlocks);
-            if (CTAS == 1) ptx::tma_load_2d(se, &map_e, full, 0, y);
-            else ptx::tma_load_2d_pair(se, &map_e, full, 0, 0, y);
           }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
@@ -200,13 +299,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (cta_rank == 0 && ptx::elect_one()) {
-      const uint32_t idesc = make_idesc<KIND>(SPARSE, p.a_fmt, kBlockM * CTAS, BLOCK_N);
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0, e_buf = 0;
       for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
+        int mt, nt;
+        tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
+        // instruction N = the columns this tile really has (a multiple of 16, of 32 for int8)
+        const int n_eff = min(BLOCK_N, (int)(p.N - (int64_t)nt * BLOCK_N));
+        const int live = min(MBLK, (int)((p.M - (int64_t)mt * MBLK * CTAS * kBlockM + CTAS * kBlockM - 1) /
+                                         (CTAS * kBlockM)));
+        const uint32_t idesc = make_idesc<KIND>(SPARSE, p.a_fmt, kBlockM * CTAS, n_eff);
         if (!bounded_wait(&sh->tmem_empty[acc], acc_phase ^ 1u, sh, p.status, 2u)) break;
         ptx::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
         bool ok = true;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!bounded_wait(&sh->full[stage], phase, sh, p.status, 3u)) { ok = false; break; }
@@ -215,30 +319,42 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           const uint32_t sb = sa + C::kABytes;
           const uint32_t se = sb + C::kBBytes;
           // metadata columns alternate between two small tensor-memory buffers from k-block to k-block
-          const uint32_t e_tmem = tmem_base + C::kECol + e_buf * 8;
+          const uint32_t e_base = tmem_base + C::kECol + e_buf * (MBLK * 8);
           e_buf ^= 1u;
           if (SPARSE) {
 #pragma unroll
-            for (int i = 0; i < C::kEBlocks; ++i)
-              ptx::tmem_cp_128x128b<CTAS>(e_tmem + 4 * i, ptx::smem_desc(se + i * 2048, false, 128));
+            for (int j = 0; j < MBLK; ++j) {
+              if (j >= live) break;
+#pragma unroll
+              for (int i = 0; i < C::kEBlocks; ++i)
+                ptx::tmem_cp_128x128b<CTAS>(e_base + j * 8 + 4 * i,
+                                            ptx::smem_desc(se + j * C::kEBlockBytes + i * 2048, false, 128));
+            }
           }
 #pragma unroll
-          for (int k = 0; k < C::kMmasPerStage; ++k) {
-            const uint32_t accumulate = (kb > 0 || k > 0) ? 1u : 0u;
-            if (SPARSE) {
-              // 32 bytes of compressed A and 64 bytes of B per instruction
-              uint64_t da = ptx::smem_desc(sa + k * 32, true, 1024);
-              uint64_t db = ptx::smem_desc(sb + (k >> 1) * C::kBRows * kAtomBytes + (k & 1) * 64, true, 1024);
-              if (KIND == 0) {
-                // one 32-bit metadata column per instruction: even-aligned address + selector
-                ptx::mma_sparse<KIND, CTAS>(d_tmem, da, db, e_tmem + (k & ~1), idesc | (uint32_t)(k & 1), accumulate);
+          for (int j = 0; j < MBLK; ++j) {
+            if (j >= live) break;
+            const uint32_t d_tmem = tmem_base + (acc * MBLK + j) * BLOCK_N;
+            const uint32_t e_tmem = e_base + j * 8;
+            const uint32_t saj = sa + j * C::kABlockBytes;
+#pragma unroll
+            for (int k = 0; k < C::kMmasPerStage; ++k) {
+              const uint32_t accumulate = (kb > 0 || k > 0) ? 1u : 0u;
+              if (SPARSE) {
+                // 32 bytes of compressed A and 64 bytes of B per instruction
+                uint64_t da = ptx::smem_desc(saj + k * 32, true, 1024);
+                uint64_t db = ptx::smem_desc(sb + (k >> 1) * C::kBRows * kAtomBytes + (k & 1) * 64, true, 1024);
+                if (KIND == 0) {
+                  // one 32-bit metadata column per instruction: even-aligned address + selector
+                  ptx::mma_sparse<KIND, CTAS>(d_tmem, da, db, e_tmem + (k & ~1), idesc | (uint32_t)(k & 1), accumulate);
+                } else {
+                  ptx::mma_sparse<KIND, CTAS>(d_tmem, da, db, e_tmem + 2 * k, idesc, accumulate);
+                }
               } else {
-                ptx::mma_sparse<KIND, CTAS>(d_tmem, da, db, e_tmem + 2 * k, idesc, accumulate);
+                uint64_t da = ptx::smem_desc(saj + (k >> 2) * kBlockM * kAtomBytes + (k & 3) * 32, true, 1024);
+                uint64_t db = ptx::smem_desc(sb + (k >> 2) * C::kBRows * kAtomBytes + (k & 3) * 32, true, 1024);
+                ptx::mma_dense<KIND, CTAS>(d_tmem, da, db, idesc, accumulate);
               }
-            } else {
-              uint64_t da = ptx::smem_desc(sa + (k >> 2) * kBlockM * kAtomBytes + (k & 3) * 32, true, 1024);
-              uint64_t db = ptx::smem_desc(sb + (k >> 2) * C::kBRows * kAtomBytes + (k & 3) * 32, true, 1024);
-              ptx::mma_dense<KIND, CTAS>(d_tmem, da, db, idesc, accumulate);
             }
           }
           // the stage may be refilled once these MMAs have read it
@@ -255,94 +371,63 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   } else {
     // ------------------------------ epilogue ------------------------------
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
-    const bool is_int = KIND == 1;
+    const int cs = elem_bytes((sp24_dtype)p.cd_type);
+    constexpr int kChunks = (BLOCK_N + 31) / 32;
     int acc = 0;
-    uint32_t acc_phase = 0;
+    uint32_t acc_phase = 0, tiles_seen = 0;
     for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
       int mt, nt;
-      tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
-      if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u)) break;
-      ptx::tc_fence_after();
-      const int64_t row = (int64_t)(mt * CTAS + (int)cta_rank) * kBlockM + q * 32 + lane;
+      tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
       const int64_t col_base = (int64_t)nt * BLOCK_N;
-      const uint32_t t_addr = tmem_base + acc * BLOCK_N + ((uint32_t)(q * 32) << 16);
-#pragma unroll 1
-      for (int c0 = 0; c0 < BLOCK_N; c0 += 32) {
-        uint32_t r[32];
-        ptx::tmem_ld_32x32b_x32(t_addr + c0, r);
-        ptx::tmem_ld_wait();
-        if (row < p.M) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int64_t col = col_base + c0 + 8 * j;
-            // N and BLOCK_N are multiples of 16, so groups of 8 columns are all-in or all-out
-            if (c0 + 8 * j >= BLOCK_N || col >= p.N) continue;
-            const int64_t off_d = row * p.ldd + col, off_c = row * p.ldc + col;
-            if (is_int) {
-              int32_t v[8];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) v[e] = (int32_t)r[8 * j + e];
-              if (p.has_c) {
-                const int4* cp = reinterpret_cast<const int4*>(static_cast<const int32_t*>(p.C) + off_c);
-                int4 c0v = cp[0], c1v = cp[1];
-                v[0] += c0v.x; v[1] += c0v.y; v[2] += c0v.z; v[3] += c0v.w;
-                v[4] += c1v.x; v[5] += c1v.y; v[6] += c1v.z; v[7] += c1v.w;
-              }
-              int4* dp = reinterpret_cast<int4*>(static_cast<int32_t*>(p.D) + off_d);
-              dp[0] = make_int4(v[0], v[1], v[2], v[3]);
-              dp[1] = make_int4(v[4], v[5], v[6], v[7]);
-            } else {
-              float v[8];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) v[e] = p.alpha * __uint_as_float(r[8 * j + e]);
-              if (p.cd_type == SP24_F32) {
-                if (p.has_c) {
-                  const float4* cp = reinterpret_cast<const float4*>(static_cast<const float*>(p.C) + off_c);
-                  float4 a = cp[0], b = cp[1];
-                  v[0] += p.beta * a.x; v[1] += p.beta * a.y; v[2] += p.beta * a.z; v[3] += p.beta * a.w;
-                  v[4] += p.beta * b.x; v[5] += p.beta * b.y; v[6] += p.beta * b.z; v[7] += p.beta * b.w;
-                }
-                float4* dp = reinterpret_cast<float4*>(static_cast<float*>(p.D) + off_d);
-                dp[0] = make_float4(v[0], v[1], v[2], v[3]);
-                dp[1] = make_float4(v[4], v[5], v[6], v[7]);
-              } else if (p.cd_type == SP24_BF16) {
-                if (p.has_c) {
-                  uint4 cv = *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.C) + off_c);
-                  const __nv_bfloat162* c2 = reinterpret_cast<const __nv_bfloat162*>(&cv);
-#pragma unroll
-                  for (int e = 0; e < 4; ++e) {
-                    float2 f = __bfloat1622float2(c2[e]);
-                    v[2 * e] += p.beta * f.x;
-                    v[2 * e + 1] += p.beta * f.y;
-                  }
-                }
-                uint4 ov;
-                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) o2[e] = __float22bfloat162_rn(make_float2(v[2 * e], v[2 * e + 1]));
-                *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.D) + off_d) = ov;
-              } else {
-                if (p.has_c) {
-                  uint4 cv = *reinterpret_cast<const uint4*>(static_cast<const __half*>(p.C) + off_c);
-                  const __half2* c2 = reinterpret_cast<const __half2*>(&cv);
-#pragma unroll
-                  for (int e = 0; e < 4; ++e) {
-                    float2 f = __half22float2(c2[e]);
-                    v[2 * e] += p.beta * f.x;
-                    v[2 * e + 1] += p.beta * f.y;
-                  }
-                }
-                uint4 ov;
-                __half2* o2 = reinterpret_cast<__half2*>(&ov);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) o2[e] = __float22half2_rn(make_float2(v[2 * e], v[2 * e + 1]));
-                *reinterpret_cast<uint4*>(static_cast<__half*>(p.D) + off_d) = ov;
-              }
-            }
-          }
+      const int n_eff = min(BLOCK_N, (int)(p.N - col_base));
+      const int64_t row_first = ((int64_t)mt * MBLK * CTAS + (int)cta_rank) * kBlockM + q * 32 + lane;
+      ++tiles_seen;
+      if (p.has_c) {
+        // Shortly before the main loop ends, ask the L2 for this thread's rows of C, so that the
+        // loads below are L2 hits.  The wait is only a hint and gives up after a while.
+        for (uint32_t spin = 0; sh->c_hint_tiles < tiles_seen && spin < (1u << 22) && !sh->abort; ++spin) __nanosleep(64);
+        for (int j = 0; j < MBLK; ++j) {
+          const int64_t row = row_first + (int64_t)j * CTAS * kBlockM;
+          if (row >= p.M) break;
+          const uint8_t* cp = static_cast<const uint8_t*>(p.C) + (row * p.ldc + col_base) * cs;
+          for (int off = 0; off < n_eff * cs; off += 128)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(cp + off));
         }
       }
-      // accumulator drained: hand it back to the MMA issuer (CTA 0 of the pair)
+      // C runs two chunks ahead of its use, the accumulator columns one chunk ahead
+      uint4 c_cur[8], c_nxt[8], c_far[8];
+      if (p.has_c && row_first < p.M) {
+        load_c_chunk(c_cur, p, cs, row_first, col_base, n_eff);
+        if (kChunks > 1 && 32 < n_eff) load_c_chunk(c_nxt, p, cs, row_first, col_base + 32, n_eff - 32);
+      }
+      if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u)) break;
+      ptx::tc_fence_after();
+      uint32_t r_next[32];
+      ptx::tmem_ld_32x32b_x32(tmem_base + (acc * MBLK) * BLOCK_N + ((uint32_t)(q * 32) << 16), r_next);
+      constexpr int kIters = MBLK * kChunks;
+#pragma unroll 1
+      for (int it = 0; it < kIters; ++it) {
+        const int j = it / kChunks, ch = it - j * kChunks;
+        const int64_t row = row_first + (int64_t)j * CTAS * kBlockM;
+        uint32_t r[32];
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) r[e] = r_next[e];
+        if (it + 1 < kIters) {
+          const int jn = (it + 1) / kChunks, chn = (it + 1) - jn * kChunks;
+          ptx::tmem_ld_32x32b_x32(tmem_base + (acc * MBLK + jn) * BLOCK_N + chn * 32 + ((uint32_t)(q * 32) << 16), r_next);
+        }
+        if (it + 2 < kIters && p.has_c) {
+          const int jf = (it + 2) / kChunks, chf = (it + 2) - jf * kChunks;
+          const int64_t rowf = row_first + (int64_t)jf * CTAS * kBlockM;
+          if (rowf < p.M && chf * 32 < n_eff) load_c_chunk(c_far, p, cs, rowf, col_base + chf * 32, n_eff - chf * 32);
+        }
+        const int cols_valid = min(32, n_eff - ch * 32);
+        if (row < p.M && cols_valid > 0) store_chunk<KIND>(r, c_cur, p, row, col_base + ch * 32, cols_valid);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { c_cur[e] = c_nxt[e]; c_nxt[e] = c_far[e]; }
+      }
+      // accumulators drained: hand them back to the MMA issuer (CTA 0 of the pair)
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) {
@@ -415,13 +500,13 @@ int sm_count() {
   return n;
 }
 
-template <int KIND, bool SPARSE, int BLOCK_N, int CTAS>
+template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK>
 sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* A, const void* meta, const void* B,
                    cudaStream_t stream) {
-  using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS>;
+  using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS, MBLK>;
   GemmParams p = base;
   const int es = KIND == 0 ? 2 : 1;
-  const int tile_m = kBlockM * CTAS;
+  const int tile_m = kBlockM * CTAS * MBLK;
   p.m_tiles = (int)((d->M + tile_m - 1) / tile_m);
   p.n_tiles = (int)((d->N + BLOCK_N - 1) / BLOCK_N);
   p.k_blocks = (int)((d->K + C::kKPerStage - 1) / C::kKPerStage);
@@ -440,7 +525,7 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
   } else {
     map_e = map_a;
   }
-  auto kernel = gemm_kernel<KIND, SPARSE, BLOCK_N, CTAS>;
+  auto kernel = gemm_kernel<KIND, SPARSE, BLOCK_N, CTAS, MBLK>;
   SP24_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
   const int tiles = p.m_tiles * p.n_tiles;
   int clusters = sm_count() / CTAS;
@@ -533,25 +618,37 @@ extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, con
   p.has_c = has_c ? 1 : 0;
   const bool sparse = !d->a_is_dense;
   const bool i8 = d->ab_type == SP24_I8;
-  // Tile choice: a pair of CTAs on 256 x 240 tiles (two accumulators fit tensor memory, so the
-  // epilogue overlaps the next tile's main loop) once the problem has enough of them to occupy
-  // the pairs; single CTAs on 128 x 128 tiles otherwise.  SP24_TILE=<ctas>x<block_n> overrides.
-  int ctas = (d->M >= 256 && (d->M / 256) * ((d->N + 239) / 240) >= 32) ? 2 : 1;
-  int block_n = ctas == 2 ? 240 : 128;
+  // Tile choice.  Large problems (at least six waves of tiles): a pair of CTAs with two m-blocks
+  // each, 512 x 224 tiles: least operand traffic per flop.  Medium: a pair with one m-block, 256 x 240
+  // (224 columns for int8, whose pair MMAs need N % 32 == 0), epilogue overlapped.  Small: single
+  // CTAs, 128 x 128.
+  // SP24_TILE=<ctas>x<block_n>x<mblk> overrides (benchmarking).
+  const int wide_n = i8 ? 224 : 240;
+  const int64_t n_tiles = (d->N + wide_n - 1) / wide_n, n_tiles_224 = (d->N + 223) / 224;
+  int ctas = 1, block_n = 128, mblk = 1;
+  if (d->M >= 512 && (d->M / 512) * n_tiles_224 >= 444) { ctas = 2; block_n = 224; mblk = 2; }
+  else if (d->M >= 256 && (d->M / 256) * n_tiles >= 32) { ctas = 2; block_n = wide_n; mblk = 1; }
+  p.band = 16 / mblk;
   if (const char* env = getenv("SP24_TILE")) {
-    int c = 0, n = 0;
-    if (sscanf(env, "%dx%d", &c, &n) == 2) { ctas = c; block_n = n; }
+    int c = 0, n = 0, m = 1;
+    if (sscanf(env, "%dx%dx%d", &c, &n, &m) >= 2) { ctas = c; block_n = n; mblk = m; }
   }
-#define SP24_DISPATCH(CT, BN)                                                                              \
-  if (ctas == CT && block_n == BN) {                                                                       \
-    if (!i8) return sparse ? launch<0, true, BN, CT>(d, p, A, meta, B, s) : launch<0, false, BN, CT>(d, p, A, meta, B, s); \
-    return sparse ? launch<1, true, BN, CT>(d, p, A, meta, B, s) : launch<1, false, BN, CT>(d, p, A, meta, B, s);          \
+  if (const char* env = getenv("SP24_BAND")) {
+    int b = atoi(env);
+    if (b > 0) p.band = b;
   }
-  SP24_DISPATCH(1, 128)
-  SP24_DISPATCH(2, 256)
-  SP24_DISPATCH(2, 240)
-  SP24_DISPATCH(2, 224)
-  SP24_DISPATCH(2, 192)
+#define SP24_DISPATCH(CT, BN, MB)                                                                            \
+  if (ctas == CT && block_n == BN && mblk == MB) {                                                           \
+    if (!i8) return sparse ? launch<0, true, BN, CT, MB>(d, p, A, meta, B, s) : launch<0, false, BN, CT, MB>(d, p, A, meta, B, s); \
+    return sparse ? launch<1, true, BN, CT, MB>(d, p, A, meta, B, s) : launch<1, false, BN, CT, MB>(d, p, A, meta, B, s);          \
+  }
+  SP24_DISPATCH(1, 128, 1)
+  SP24_DISPATCH(2, 240, 1)
+  SP24_DISPATCH(2, 224, 1)
+  SP24_DISPATCH(2, 240, 2)
+  SP24_DISPATCH(2, 224, 2)
+  SP24_DISPATCH(2, 192, 2)
+  SP24_DISPATCH(2, 256, 1)
 #undef SP24_DISPATCH
   return SP24_ERR_UNSUPPORTED;
 }

@@ -287,6 +287,58 @@ def run_ours(args, cfg):
         "speedup_vs_dense_variant": dense_ms / gemm_ms,
     }
 
+    # ---- context: cuBLAS dense on the same pruned matrix (a library call, not part of the path) ----
+    if ab != "i8":
+        torch_ms = time_call(lambda: torch.matmul(A_pruned, Bt.t()), reps=3)
+        kernels["context_torch_matmul_dense_ms"] = torch_ms
+        kernels["context_torch_matmul_dense_tflops"] = flop / (torch_ms * 1e-3) / 1e12
+        kernels["speedup_vs_torch_matmul_dense"] = torch_ms / gemm_ms
+
+    # ---- the other configurations (GEMM only, L2 flushed between repetitions) ----
+    others = {}
+    if world == 1 and not args.no_other_configs and not args.rows:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+        def time_flushed(fn, reps=7):
+            fn()
+            ts = []
+            for _ in range(reps):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            return float(np.median(ts))
+
+        for name in inputs.CONFIG_ORDER:
+            oc = inputs.CONFIGS[name]
+            if name == cfg.name:
+                continue
+            oA = dev_tensor(inputs.gen_A(oc), oc.ab_type)
+            if oc.conv is not None:
+                x = dev_tensor(inputs.gen_conv_input(oc), oc.ab_type)
+                im2col_ms = time_flushed(lambda: sp.im2col_nhwc_3x3(x), reps=3)
+                oB = sp.im2col_nhwc_3x3(x)
+            else:
+                im2col_ms = None
+                oB = dev_tensor(inputs.gen_Bt(oc), oc.ab_type)
+            ovals, ometa, _ = sp.compress(oA)
+            opruned = sp.prune(oA)
+            oD = torch.empty((oc.M, oc.N), dtype=tdt[oc.cd_type], device=dev)
+            s_ms = time_flushed(lambda: sp.gemm(ovals, ometa, oB, out=oD, cd=oc.cd_type, ws=ws))
+            d_ms = time_flushed(lambda: sp.gemm(opruned, None, oB, out=oD, cd=oc.cd_type, a_is_dense=True, ws=ws))
+            peak = 2.0 * peaks["bf16_tflops"] * (2.0 if oc.ab_type == "i8" else 1.0)
+            others[name] = {"M": oc.M, "N": oc.N, "K": oc.K, "ab": oc.ab_type, "gemm_ms": s_ms,
+                            "gemm_dense_equiv_tflops": oc.dense_equiv_flop / (s_ms * 1e-3) / 1e12,
+                            "frac_of_2x_measured_dense": oc.dense_equiv_flop / (s_ms * 1e-3) / 1e12 / peak,
+                            "dense_variant_ms": d_ms, "speedup_vs_dense_variant": d_ms / s_ms}
+            if im2col_ms is not None:
+                others[name]["im2col_ms"] = im2col_ms
+            del oA, oB, ovals, ometa, opruned, oD
+        del flush
+
     # ---- end to end through the host-buffer entry point (rank-local) ----
     import ctypes
     e2e = None
@@ -324,7 +376,7 @@ def run_ours(args, cfg):
 
     if rank != 0:
         return
-    kernel_name = "sp24_gemm (tcgen05.mma.sp, 2-CTA 256x240 tiles)"
+    kernel_name = "sp24_gemm (tcgen05.mma.sp, CTA pairs, 512x224 tiles)"
     roofline = {
         "kernel": kernel_name, "bound": "tensor", "achieved": gemm_tflops, "peak": sparse_peak, "unit": UNIT,
         "frac": gemm_tflops / sparse_peak,
@@ -348,7 +400,7 @@ def run_ours(args, cfg):
                    "cd_type": cd, "tokens_per_gpu": N, "parallelism": f"replicated weight, tokens sharded x{world}",
                    "l2": "inputs larger than L2 (A 1.2 GB, vals 0.6 GB, B 0.2 GB per step)"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * args.steps, "roofline": roofline, "cpu_baseline": cpu,
-        "kernels": kernels,
+        "kernels": kernels, "other_configs": others,
     }
     print(json.dumps(line))
 
@@ -362,6 +414,7 @@ def main():
     ap.add_argument("--config", default="gpt3_ffn_bf16", choices=inputs.CONFIG_ORDER)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the GEMM timings of the other configurations")
     ap.add_argument("--rows", type=int, default=0,
                     help="use only the first ROWS rows of A (a smaller case of the same kernel for ncu captures)")
     args = ap.parse_args()

@@ -70,23 +70,30 @@ struct Cfg {
   static constexpr int kEBytes = MBLK * kEBlockBytes;
   static constexpr int kEAlloc = (kEBytes + 1023) / 1024 * 1024;
   static constexpr int kStageBytes = kABytes + kBBytes + kEAlloc;
-  static constexpr int kStages = (216 * 1024) / kStageBytes > 8 ? 8 : (216 * 1024) / kStageBytes;
-  static constexpr int kAccStages = MBLK == 2 ? 1 : ((2 * BLOCK_N + 32 <= (int)kTmemCols) ? 2 : 1);
+  // shared memory: [stage ring | epilogue staging | barriers]; 1 KB of slack for the 1024-byte alignment
+  static constexpr int kSmemLimit = 232448 - 1024 - 512;
+  static constexpr int kStagesFit = (kSmemLimit - 16384) / kStageBytes;
+  static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
+  static constexpr int kEpiBytes = (kSmemLimit - kStages * kStageBytes >= 32768) ? 32768 : 16384;  // all 4 warps
+  static constexpr int kAccStages = MBLK == 2 ? 1 : ((2 * BLOCK_N + (SPARSE ? 32 : 0) <= (int)kTmemCols) ? 2 : 1);
   static constexpr int kECol = kAccStages * MBLK * BLOCK_N;        // first metadata column in tensor memory
   static constexpr int kMmasPerStage = SPARSE ? 4 : 4 * kBBoxes;   // per m-block
   static constexpr int kKPerStage = (KIND == 0 ? 64 : 128) * kBBoxes;  // logical K per stage
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
   static_assert(kStages >= 2, "need at least two stages");
+  static_assert(BLOCK_N % 32 == 0, "the epilogue moves 32-column boxes");
   static_assert(kStageBytes % 1024 == 0, "stages must keep the 1024-byte alignment of the atoms");
   static_assert(kECol + (SPARSE ? 2 * MBLK * 8 : 0) <= (int)kTmemCols, "tensor memory overflow");
 };
 
 struct Shared {
   uint64_t full[8], empty[8], tmem_full[2], tmem_empty[2];
+  uint64_t c_full[4][4];           // per epilogue warp and staging buffer: C box has landed
   uint32_t tmem_base;
   volatile uint32_t abort;
   volatile uint32_t c_hint_tiles;  // tiles whose main loop is close enough to its end to fetch C into the L2
 };
+static_assert(sizeof(Shared) <= 512, "barrier block");
 
 __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, Shared* sh, uint32_t* status,
                                              uint32_t code) {
@@ -129,74 +136,70 @@ __device__ __forceinline__ uint32_t make_idesc(bool sparse, int a_fmt, int m, in
   return d;                                        // both operands K-major, no negate, no saturate
 }
 
-// ---- epilogue helpers: one chunk = 32 consecutive columns of one row ---------------------------
-// C for the chunk, fetched one chunk ahead of its use: 64 bytes (16-bit types) or 128 bytes per thread.
-__device__ __forceinline__ void load_c_chunk(uint4 (&c)[8], const GemmParams& p, int cs, int64_t row, int64_t col,
-                                             int cols_valid) {
-  const uint8_t* base = static_cast<const uint8_t*>(p.C) + (row * p.ldc + col) * cs;
-  const int vecs = 2 * cs;  // 16-byte vectors per chunk: 4 for 2-byte, 8 for 4-byte types
-  const int per_vec = 16 / cs;
-#pragma unroll
-  for (int v = 0; v < 8; ++v)
-    if (v < vecs && v * per_vec < cols_valid) c[v] = __ldg(reinterpret_cast<const uint4*>(base) + v);
+// ---- epilogue helpers ----------------------------------------------------------------------------
+// A staging buffer holds one 32-row x 32-column box of C / D in the layout the TMA uses: rows of 64
+// bytes with the 64-byte swizzle (2-byte types) or rows of 128 bytes with the 128-byte swizzle
+// (4-byte types).  16-byte unit v of row r sits at unit v ^ ((r >> 1) & 3), resp. v ^ (r & 7), which
+// also keeps the row-per-thread accesses below free of bank conflicts.
+__device__ __forceinline__ uint4* staged_unit(uint8_t* buf, int cs, int row, int v) {
+  return cs == 2 ? reinterpret_cast<uint4*>(buf + row * 64 + ((v ^ ((row >> 1) & 3)) << 4))
+                 : reinterpret_cast<uint4*>(buf + row * 128 + ((v ^ (row & 7)) << 4));
 }
 
+// This thread's row of the box: out = alpha * acc + beta * c, written over c in the staging buffer.
 template <int KIND>
-__device__ __forceinline__ void store_chunk(const uint32_t (&r)[32], const uint4 (&c)[8], const GemmParams& p,
-                                            int64_t row, int64_t col, int cols_valid) {
+__device__ __forceinline__ void convert_row(const uint32_t (&r)[32], uint8_t* buf, int lane, const GemmParams& p) {
   if (KIND == 1) {
-    int32_t* dp = static_cast<int32_t*>(p.D) + row * p.ldd + col;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      if (4 * j >= cols_valid) break;
-      int4 v = make_int4((int)r[4 * j], (int)r[4 * j + 1], (int)r[4 * j + 2], (int)r[4 * j + 3]);
-      if (p.has_c) { v.x += (int)c[j].x; v.y += (int)c[j].y; v.z += (int)c[j].z; v.w += (int)c[j].w; }
-      reinterpret_cast<int4*>(dp)[j] = v;
+    for (int v = 0; v < 8; ++v) {
+      uint4* u = staged_unit(buf, 4, lane, v);
+      uint4 o = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+      if (p.has_c) { uint4 c = *u; o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w; }
+      *u = o;
     }
   } else if (p.cd_type == SP24_F32) {
-    float* dp = static_cast<float*>(p.D) + row * p.ldd + col;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      if (4 * j >= cols_valid) break;
-      float4 v = make_float4(p.alpha * __uint_as_float(r[4 * j]), p.alpha * __uint_as_float(r[4 * j + 1]),
-                             p.alpha * __uint_as_float(r[4 * j + 2]), p.alpha * __uint_as_float(r[4 * j + 3]));
+    for (int v = 0; v < 8; ++v) {
+      uint4* u = staged_unit(buf, 4, lane, v);
+      float4 o = make_float4(p.alpha * __uint_as_float(r[4 * v]), p.alpha * __uint_as_float(r[4 * v + 1]),
+                             p.alpha * __uint_as_float(r[4 * v + 2]), p.alpha * __uint_as_float(r[4 * v + 3]));
       if (p.has_c) {
-        v.x += p.beta * __uint_as_float(c[j].x); v.y += p.beta * __uint_as_float(c[j].y);
-        v.z += p.beta * __uint_as_float(c[j].z); v.w += p.beta * __uint_as_float(c[j].w);
+        float4 c = *reinterpret_cast<float4*>(u);
+        o.x += p.beta * c.x; o.y += p.beta * c.y; o.z += p.beta * c.z; o.w += p.beta * c.w;
       }
-      reinterpret_cast<float4*>(dp)[j] = v;
+      *reinterpret_cast<float4*>(u) = o;
     }
   } else {
     const bool bf = p.cd_type == SP24_BF16;
-    uint16_t* dp = static_cast<uint16_t*>(p.D) + row * p.ldd + col;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (8 * j >= cols_valid) break;
-      float v[8];
+    for (int v = 0; v < 4; ++v) {
+      uint4* u = staged_unit(buf, 2, lane, v);
+      float f[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) v[e] = p.alpha * __uint_as_float(r[8 * j + e]);
+      for (int e = 0; e < 8; ++e) f[e] = p.alpha * __uint_as_float(r[8 * v + e]);
       if (p.has_c) {
-        const uint32_t cw[4] = {c[j].x, c[j].y, c[j].z, c[j].w};
+        uint4 c = *u;
+        const uint32_t cw[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          float2 f = bf ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&cw[e]))
+          float2 g = bf ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&cw[e]))
                         : __half22float2(*reinterpret_cast<const __half2*>(&cw[e]));
-          v[2 * e] += p.beta * f.x;
-          v[2 * e + 1] += p.beta * f.y;
+          f[2 * e] += p.beta * g.x;
+          f[2 * e + 1] += p.beta * g.y;
         }
       }
       uint32_t ow[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         if (bf) {
-          __nv_bfloat162 o = __float22bfloat162_rn(make_float2(v[2 * e], v[2 * e + 1]));
+          __nv_bfloat162 o = __float22bfloat162_rn(make_float2(f[2 * e], f[2 * e + 1]));
           ow[e] = *reinterpret_cast<uint32_t*>(&o);
         } else {
-          __half2 o = __float22half2_rn(make_float2(v[2 * e], v[2 * e + 1]));
+          __half2 o = __float22half2_rn(make_float2(f[2 * e], f[2 * e + 1]));
           ow[e] = *reinterpret_cast<uint32_t*>(&o);
         }
       }
-      reinterpret_cast<uint4*>(dp)[j] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+      *u = make_uint4(ow[0], ow[1], ow[2], ow[3]);
     }
   }
 }
@@ -204,12 +207,14 @@ __device__ __forceinline__ void store_chunk(const uint32_t (&r)[32], const uint4
 template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK>
 __global__ void __launch_bounds__(kNumThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            const __grid_constant__ CUtensorMap map_e, const GemmParams p) {
+            const __grid_constant__ CUtensorMap map_e, const __grid_constant__ CUtensorMap map_c,
+            const __grid_constant__ CUtensorMap map_d, const GemmParams p) {
   using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS, MBLK>;
   extern __shared__ uint8_t smem_raw[];
   // Operand atoms need 1024-byte alignment for the 128-byte swizzle.
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  Shared* sh = reinterpret_cast<Shared*>(smem + C::kStages * C::kStageBytes);
+  uint8_t* epi = smem + C::kStages * C::kStageBytes;
+  Shared* sh = reinterpret_cast<Shared*>(epi + C::kEpiBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t cta_rank = CTAS == 2 ? ptx::cluster_ctarank() : 0;
@@ -225,12 +230,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       ptx::mbar_init(&sh->tmem_full[a], 1);
       ptx::mbar_init(&sh->tmem_empty[a], 4 * CTAS);  // one arrival per epilogue warp of the pair
     }
+    for (int w = 0; w < 4; ++w)
+      for (int b = 0; b < 4; ++b) ptx::mbar_init(&sh->c_full[w][b], 1);
     sh->abort = 0;
     sh->c_hint_tiles = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&map_a);
     ptx::prefetch_tensormap(&map_b);
     if (SPARSE) ptx::prefetch_tensormap(&map_e);
+    if (p.has_c) ptx::prefetch_tensormap(&map_c);
+    ptx::prefetch_tensormap(&map_d);
   }
   if (warp == 1) {
     ptx::tmem_alloc<CTAS>(&sh->tmem_base, kTmemCols);
@@ -370,63 +379,96 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     }
   } else {
     // ------------------------------ epilogue ------------------------------
+    // Each warp owns 32 accumulator rows and walks its tiles in 32 x 32 boxes: TMA load of the C box
+    // (if beta != 0) into a staging buffer a few boxes ahead, tcgen05.ld of the accumulator columns,
+    // convert in place, TMA store of the D box.  Boxes outside the matrix are clipped by the TMA.
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
     const int cs = elem_bytes((sp24_dtype)p.cd_type);
-    constexpr int kChunks = (BLOCK_N + 31) / 32;
-    int acc = 0;
-    uint32_t acc_phase = 0, tiles_seen = 0;
-    for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
+    const int buf_bytes = 1024 * cs;
+    const int nbuf = C::kEpiBytes / 4 / buf_bytes;  // staging buffers of this warp: 1, 2 or 4
+    const int ahead = nbuf > 1 ? nbuf - 1 : 1;      // boxes the C loads run ahead
+    uint8_t* my_bufs = epi + q * (C::kEpiBytes / 4);
+    constexpr int kSub = BLOCK_N / 32;
+    constexpr int kIters = MBLK * kSub;
+
+    // box `it` of tile `t`: first row / column and whether any of it lies inside the matrix
+    auto box_of = [&](int t, int it, int& row0, int& col0) -> bool {
       int mt, nt;
       tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
-      const int64_t col_base = (int64_t)nt * BLOCK_N;
-      const int n_eff = min(BLOCK_N, (int)(p.N - col_base));
-      const int64_t row_first = ((int64_t)mt * MBLK * CTAS + (int)cta_rank) * kBlockM + q * 32 + lane;
-      ++tiles_seen;
-      if (p.has_c) {
-        // Shortly before the main loop ends, ask the L2 for this thread's rows of C, so that the
-        // loads below are L2 hits.  The wait is only a hint and gives up after a while.
-        for (uint32_t spin = 0; sh->c_hint_tiles < tiles_seen && spin < (1u << 22) && !sh->abort; ++spin) __nanosleep(64);
-        for (int j = 0; j < MBLK; ++j) {
-          const int64_t row = row_first + (int64_t)j * CTAS * kBlockM;
-          if (row >= p.M) break;
-          const uint8_t* cp = static_cast<const uint8_t*>(p.C) + (row * p.ldc + col_base) * cs;
-          for (int off = 0; off < n_eff * cs; off += 128)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(cp + off));
+      const int j = it / kSub, sc = it - j * kSub;
+      row0 = ((mt * MBLK + j) * CTAS + (int)cta_rank) * kBlockM + q * 32;
+      col0 = nt * BLOCK_N + sc * 32;
+      return row0 < p.M && col0 < p.N;
+    };
+    // cursor of the C loads over the same stream of boxes, `ahead` live boxes in front of the consumer
+    int pf_t = cluster_id, pf_it = 0;
+    uint32_t pf_seq = 0;
+    auto issue_c_load = [&]() {  // lane 0 only: load the next live box of the stream, if any
+      while (pf_t < num_tiles) {
+        int row0, col0;
+        const bool live_box = box_of(pf_t, pf_it, row0, col0);
+        if (++pf_it == kIters) { pf_it = 0; pf_t += num_clusters; }
+        if (live_box) {
+          const int b = pf_seq % nbuf;
+          ptx::mbar_expect_tx(&sh->c_full[q][b], (uint32_t)buf_bytes);
+          ptx::tma_load_2d(my_bufs + b * buf_bytes, &map_c, &sh->c_full[q][b], col0, row0);
+          ++pf_seq;
+          return;
         }
       }
-      // C runs two chunks ahead of its use, the accumulator columns one chunk ahead
-      uint4 c_cur[8], c_nxt[8], c_far[8];
-      if (p.has_c && row_first < p.M) {
-        load_c_chunk(c_cur, p, cs, row_first, col_base, n_eff);
-        if (kChunks > 1 && 32 < n_eff) load_c_chunk(c_nxt, p, cs, row_first, col_base + 32, n_eff - 32);
+    };
+    if (p.has_c && lane == 0)
+      for (int i = 0; i < ahead; ++i) issue_c_load();
+
+    int acc = 0;
+    uint32_t acc_phase = 0, seq = 0, tiles_seen = 0;
+    for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
+      ++tiles_seen;
+      if (p.has_c && lane == 0) {
+        // Shortly before the main loop ends, ask the L2 for this warp's boxes of C so that the loads
+        // above are L2 hits.  The wait is only a hint and gives up after a while.
+        for (uint32_t spin = 0; sh->c_hint_tiles < tiles_seen && spin < (1u << 20) && !sh->abort; ++spin) __nanosleep(128);
+        for (int it = 0; it < kIters; ++it) {
+          int row0, col0;
+          if (box_of(t, it, row0, col0)) ptx::tma_prefetch_2d(&map_c, col0, row0);
+        }
       }
       if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u)) break;
       ptx::tc_fence_after();
       uint32_t r_next[32];
-      ptx::tmem_ld_32x32b_x32(tmem_base + (acc * MBLK) * BLOCK_N + ((uint32_t)(q * 32) << 16), r_next);
-      constexpr int kIters = MBLK * kChunks;
+      const uint32_t t_acc = tmem_base + (acc * MBLK) * BLOCK_N + ((uint32_t)(q * 32) << 16);
+      ptx::tmem_ld_32x32b_x32(t_acc, r_next);
+      bool ok = true;
 #pragma unroll 1
       for (int it = 0; it < kIters; ++it) {
-        const int j = it / kChunks, ch = it - j * kChunks;
-        const int64_t row = row_first + (int64_t)j * CTAS * kBlockM;
         uint32_t r[32];
         ptx::tmem_ld_wait();
 #pragma unroll
         for (int e = 0; e < 32; ++e) r[e] = r_next[e];
         if (it + 1 < kIters) {
-          const int jn = (it + 1) / kChunks, chn = (it + 1) - jn * kChunks;
-          ptx::tmem_ld_32x32b_x32(tmem_base + (acc * MBLK + jn) * BLOCK_N + chn * 32 + ((uint32_t)(q * 32) << 16), r_next);
+          const int jn = (it + 1) / kSub, scn = (it + 1) - jn * kSub;
+          ptx::tmem_ld_32x32b_x32(t_acc + jn * BLOCK_N + scn * 32, r_next);
         }
-        if (it + 2 < kIters && p.has_c) {
-          const int jf = (it + 2) / kChunks, chf = (it + 2) - jf * kChunks;
-          const int64_t rowf = row_first + (int64_t)jf * CTAS * kBlockM;
-          if (rowf < p.M && chf * 32 < n_eff) load_c_chunk(c_far, p, cs, rowf, col_base + chf * 32, n_eff - chf * 32);
+        int row0, col0;
+        if (!box_of(t, it, row0, col0)) continue;  // same answer for the whole warp
+        const int b = seq % nbuf;
+        uint8_t* buf = my_bufs + b * buf_bytes;
+        if (p.has_c && !bounded_wait(&sh->c_full[q][b], (seq / nbuf) & 1u, sh, p.status, 5u)) { ok = false; break; }
+        convert_row<KIND>(r, buf, lane, p);
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          ptx::tma_store_2d(&map_d, buf, col0, row0);
+          ptx::bulk_commit_group();
+          // the buffer used one box earlier is free once its store has read it
+          if (nbuf > 1) ptx::bulk_wait_group_read<1>();
+          else ptx::bulk_wait_group_read<0>();
+          if (p.has_c) issue_c_load();
         }
-        const int cols_valid = min(32, n_eff - ch * 32);
-        if (row < p.M && cols_valid > 0) store_chunk<KIND>(r, c_cur, p, row, col_base + ch * 32, cols_valid);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) { c_cur[e] = c_nxt[e]; c_nxt[e] = c_far[e]; }
+        __syncwarp();
+        ++seq;
       }
+      if (!ok) break;
       // accumulators drained: hand them back to the MMA issuer (CTA 0 of the pair)
       ptx::tc_fence_before();
       __syncwarp();
@@ -436,6 +478,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       }
       if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
     }
+    if (lane == 0) ptx::bulk_wait_group_read<0>();  // staging buffers must outlive the stores that read them
   }
 
   // ------------------------------ teardown ------------------------------
@@ -476,16 +519,18 @@ EncodeTiledFn encode_fn() {
 // 2-D tensor map over a row-major (rows x cols) array of `es`-byte elements with `ld_bytes`
 // between rows; box = box_cols x box_rows elements.
 sp24_status make_map(CUtensorMap* map, const void* base, int es, uint64_t rows, uint64_t cols, uint64_t ld_bytes,
-                     uint32_t box_cols, uint32_t box_rows, bool swizzle128) {
+                     uint32_t box_cols, uint32_t box_rows, int swizzle_bytes) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return SP24_ERR_CUDA;
   cuuint64_t dims[2] = {cols, rows};
   cuuint64_t strides[1] = {ld_bytes};
   cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUtensorMapDataType dt = es == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
-  CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+  CUtensorMapDataType dt = es == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
+                                   : (es == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
+  CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                               : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE);
+  CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? SP24_OK : SP24_ERR_CUDA;
 }
@@ -514,16 +559,27 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
   CUtensorMap map_a, map_b, map_e;
   const uint32_t atom_elems = kAtomBytes / es;
   const uint64_t a_cols = SPARSE ? d->K / 2 : d->K;
-  sp24_status st = make_map(&map_a, A, es, d->M, a_cols, d->lda * es, atom_elems, kBlockM, true);
+  sp24_status st = make_map(&map_a, A, es, d->M, a_cols, d->lda * es, atom_elems, kBlockM, 128);
   if (st != SP24_OK) return st;
-  st = make_map(&map_b, B, es, d->N, d->K, d->ldb * es, atom_elems, C::kBRows, true);
+  st = make_map(&map_b, B, es, d->N, d->K, d->ldb * es, atom_elems, C::kBRows, 128);
   if (st != SP24_OK) return st;
   if (SPARSE) {
     uint64_t meta_rows = (uint64_t)((d->M + 127) / 128) * p.meta_kb * 16;  // rows of 128 bytes
-    st = make_map(&map_e, meta, 1, meta_rows, 128, 128, 128, 16 * C::kEBlocks, false);
+    st = make_map(&map_e, meta, 1, meta_rows, 128, 128, 128, 16 * C::kEBlocks, 0);
     if (st != SP24_OK) return st;
   } else {
     map_e = map_a;
+  }
+  // C and D move in 32 x 32 boxes whose rows are 64 bytes (2-byte types) or 128 bytes (4-byte types)
+  CUtensorMap map_c, map_d;
+  const int cs = elem_bytes(d->cd_type);
+  st = make_map(&map_d, p.D, cs, d->M, d->N, d->ldd * cs, 32, 32, 32 * cs);
+  if (st != SP24_OK) return st;
+  if (p.has_c) {
+    st = make_map(&map_c, p.C, cs, d->M, d->N, d->ldc * cs, 32, 32, 32 * cs);
+    if (st != SP24_OK) return st;
+  } else {
+    map_c = map_d;
   }
   auto kernel = gemm_kernel<KIND, SPARSE, BLOCK_N, CTAS, MBLK>;
   SP24_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
@@ -542,7 +598,7 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  SP24_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_e, p));
+  SP24_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_e, map_c, map_d, p));
   return SP24_OK;
 }
 
@@ -619,15 +675,14 @@ extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, con
   const bool sparse = !d->a_is_dense;
   const bool i8 = d->ab_type == SP24_I8;
   // Tile choice.  Large problems (at least six waves of tiles): a pair of CTAs with two m-blocks
-  // each, 512 x 224 tiles: least operand traffic per flop.  Medium: a pair with one m-block, 256 x 240
-  // (224 columns for int8, whose pair MMAs need N % 32 == 0), epilogue overlapped.  Small: single
-  // CTAs, 128 x 128.
+  // each, 512 x 224 tiles: least operand traffic per flop.  Medium: a pair with one m-block, 256 x 224,
+  // epilogue overlapped.  Small: single CTAs, 128 x 128.  (224: two fp32 accumulators plus the
+  // metadata columns fit the 512 columns of tensor memory, and 224 is a multiple of 32.)
   // SP24_TILE=<ctas>x<block_n>x<mblk> overrides (benchmarking).
-  const int wide_n = i8 ? 224 : 240;
-  const int64_t n_tiles = (d->N + wide_n - 1) / wide_n, n_tiles_224 = (d->N + 223) / 224;
+  const int64_t n_tiles = (d->N + 223) / 224;
   int ctas = 1, block_n = 128, mblk = 1;
-  if (d->M >= 512 && (d->M / 512) * n_tiles_224 >= 444) { ctas = 2; block_n = 224; mblk = 2; }
-  else if (d->M >= 256 && (d->M / 256) * n_tiles >= 32) { ctas = 2; block_n = wide_n; mblk = 1; }
+  if (d->M >= 512 && (d->M / 512) * n_tiles >= 444) { ctas = 2; block_n = 224; mblk = 2; }
+  else if (d->M >= 256 && (d->M / 256) * n_tiles >= 32) { ctas = 2; block_n = 224; mblk = 1; }
   p.band = 16 / mblk;
   if (const char* env = getenv("SP24_TILE")) {
     int c = 0, n = 0, m = 1;
@@ -643,9 +698,7 @@ extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, con
     return sparse ? launch<1, true, BN, CT, MB>(d, p, A, meta, B, s) : launch<1, false, BN, CT, MB>(d, p, A, meta, B, s);          \
   }
   SP24_DISPATCH(1, 128, 1)
-  SP24_DISPATCH(2, 240, 1)
   SP24_DISPATCH(2, 224, 1)
-  SP24_DISPATCH(2, 240, 2)
   SP24_DISPATCH(2, 224, 2)
   SP24_DISPATCH(2, 192, 2)
   SP24_DISPATCH(2, 256, 1)

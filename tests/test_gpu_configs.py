@@ -46,7 +46,8 @@ def _check_tiles(cfg, D, vals_ref, meta_ref, Bt, Cm, tiles):
             scale = abs(cfg.alpha) * oracle.gemm_abs(vals_ref, meta_ref, Bt, ab, rows=rows, cols=cols)
             beta_c = None
             if cfg.beta != 0:
-                beta_c = abs(cfg.beta) * np.abs(oracle.bits_to_float64(Cm, cd))[rows[0]:rows[1], cols[0]:cols[1]]
+                beta_c = abs(cfg.beta) * np.abs(oracle.bits_to_float64(
+                    np.ascontiguousarray(Cm[rows[0]:rows[1], cols[0]:cols[1]]), cd))
             check_fp(got, ref, scale, beta_c)
 
 

@@ -77,7 +77,8 @@ def run_case(sp, cfg, dense=False, cd=None, rows=None, cols=None, alpha=None, be
         scale = abs(alpha) * oracle.gemm_abs(vals_ref, meta_ref, Bt, ab, rows=rows, cols=cols)
         beta_c = None
         if beta != 0:
-            beta_c = abs(beta) * np.abs(oracle.bits_to_float64(Cm, cd) if cd != "f32" else Cm)[r0:r1, c0:c1]
+            csub = np.ascontiguousarray(Cm[r0:r1, c0:c1])
+            beta_c = abs(beta) * np.abs(oracle.bits_to_float64(csub, cd) if cd != "f32" else csub)
         check_fp(got, ref, scale, beta_c)
     return D
 

@@ -234,6 +234,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       for (int b = 0; b < 4; ++b) ptx::mbar_init(&sh->c_full[w][b], 1);
     sh->abort = 0;
     sh->c_hint_tiles = 0;
+    if (blockIdx.x == 0) p.status[0] = 0;  // a wait can only expire a second later
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&map_a);
     ptx::prefetch_tensormap(&map_b);
@@ -386,7 +387,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int cs = elem_bytes((sp24_dtype)p.cd_type);
     const int buf_bytes = 1024 * cs;
     const int nbuf = C::kEpiBytes / 4 / buf_bytes;  // staging buffers of this warp: 1, 2 or 4
-    const int ahead = nbuf > 1 ? nbuf - 1 : 1;      // boxes the C loads run ahead
+    const int ahead = nbuf >= 4 ? 2 : 1;            // boxes the C loads run ahead
+    // stores that may still be reading their buffer when the next buffer is claimed: with C the
+    // buffer of box seq + ahead is claimed at the end of box seq, without C that of box seq + 1
+    const int pending_ok = p.has_c ? nbuf - ahead : nbuf - 1;
     uint8_t* my_bufs = epi + q * (C::kEpiBytes / 4);
     constexpr int kSub = BLOCK_N / 32;
     constexpr int kIters = MBLK * kSub;
@@ -460,8 +464,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (lane == 0) {
           ptx::tma_store_2d(&map_d, buf, col0, row0);
           ptx::bulk_commit_group();
-          // the buffer used one box earlier is free once its store has read it
-          if (nbuf > 1) ptx::bulk_wait_group_read<1>();
+          // the buffer claimed next is free once the store that used it last has read it
+          if (pending_ok >= 3) ptx::bulk_wait_group_read<3>();
+          else if (pending_ok == 2) ptx::bulk_wait_group_read<2>();
+          else if (pending_ok == 1) ptx::bulk_wait_group_read<1>();
           else ptx::bulk_wait_group_read<0>();
           if (p.has_c) issue_c_load();
         }
@@ -661,7 +667,6 @@ extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, con
   if (d->M == 0 || d->N == 0) return SP24_OK;
   if ((st = check_arch()) != SP24_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  SP24_CUDA_CHECK(cudaMemsetAsync(workspace, 0, 16, s));
   GemmParams p = {};
   p.M = d->M; p.N = d->N; p.K = d->K;
   p.ldc = d->ldc; p.ldd = d->ldd;

@@ -205,47 +205,58 @@ __device__ __forceinline__ void count_dropped(uint32_t lost, unsigned long long*
 // 16-bit types.  Work unit: 8 columns (two groups) = one 16-byte load, 8 bytes of values and one
 // metadata byte out, so a warp reads 512 and writes 256 contiguous bytes per step.  Lanes 2j and
 // 2j+1 hold the two halves of a 16-column chunk; the even lane stores the chunk's 16 metadata bits.
-template <int UNROLL, bool COUNT>
+// HW: metadata goes straight into the tensor-core operand order.  FULL: the launch covers exactly
+// the matrix (no padding rows / columns, no ragged block), so no bounds are checked.
+template <int UNROLL, bool COUNT, bool HW, bool FULL>
 __global__ void __launch_bounds__(kThreads, 4) compress16_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
                                                               uint8_t* __restrict__ vals, int64_t row_bytes_v,
-                                                              uint8_t* __restrict__ meta, int layout, int64_t M,
-                                                              int64_t K, int64_t rows_pad, int64_t chunks_pad,
+                                                              uint8_t* __restrict__ meta, int64_t M, int64_t K,
+                                                              int64_t rows_pad, int64_t chunks_pad,
                                                               unsigned long long* dropped) {
   __shared__ uint32_t table[64];
   build_selection_table(table);
-  const int64_t halves = K >> 3, halves_pad = chunks_pad * 2, KB = chunks_pad >> 3;
-  const int64_t h0 = (int64_t)blockIdx.x * UNROLL * blockDim.x + threadIdx.x;
+  const uint32_t halves = (uint32_t)(K >> 3), halves_pad = (uint32_t)chunks_pad * 2, KB = (uint32_t)(chunks_pad >> 3);
+  const uint32_t h0 = blockIdx.x * UNROLL * blockDim.x + threadIdx.x;
+  // metadata offset of this thread's chunks inside a row: fixed for the whole kernel
+  uint32_t moff[UNROLL];
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u) {
+    const uint32_t chunk = (h0 + u * blockDim.x) >> 1;
+    moff[u] = HW ? (chunk >> 3) * 2048u + 128u * (chunk & 1u) + 4u * ((chunk >> 1) & 3u) : 2u * chunk;
+  }
   uint32_t lost = 0;
   for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows_pad;
        row += (int64_t)gridDim.y * blockDim.y) {
+    const uint8_t* xr = x + row * row_bytes_x;
+    uint8_t* vr = vals + row * row_bytes_v;
+    const uint32_t r = (uint32_t)row & 127u;
+    uint8_t* mr = HW ? meta + (row >> 7) * ((int64_t)KB * 2048) + (16u * (r & 7u) + 2u * ((r >> 3) & 1u) + 256u * (r >> 4))
+                     : meta + row * (K >> 3);
+    const bool row_live = FULL || row < M;
     uint4 in[UNROLL];
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
-      int64_t half = h0 + (int64_t)u * blockDim.x;
-      if (row < M && half < halves) in[u] = ld_stream(x + row * row_bytes_x + half * 16);
+      const uint32_t half = h0 + u * blockDim.x;
+      if (row_live && (FULL || half < halves)) in[u] = ld_stream(xr + half * 16u);
     }
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
-      int64_t half = h0 + (int64_t)u * blockDim.x;
+      const uint32_t half = h0 + u * blockDim.x;
       uint32_t mbyte = 0x44u;  // padding: positions (0, 1) in both groups
-      if (row < M && half < halves) {
-        uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
-        uint32_t out[2];
-        mbyte = 0;
-#pragma unroll
-        for (int g = 0; g < 2; ++g) {
-          uint32_t lo = w[2 * g], hi = w[2 * g + 1];
-          uint32_t e = table[selection_index(lo & 0x7FFF7FFFu, hi & 0x7FFF7FFFu)];
-          out[g] = __byte_perm(lo, hi, e >> 16);
-          mbyte |= (e & 0xFu) << (4 * g);
-          if (COUNT) lost += __popc(Group16::nonzero(lo, hi) & ~(e >> 4) & 0xFu);
-        }
-        __stcs(reinterpret_cast<uint2*>(vals + row * row_bytes_v + half * 8), make_uint2(out[0], out[1]));
+      if (row_live && (FULL || half < halves)) {
+        const uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
+        const uint32_t e0 = table[selection_index(w[0] & 0x7FFF7FFFu, w[1] & 0x7FFF7FFFu)];
+        const uint32_t e1 = table[selection_index(w[2] & 0x7FFF7FFFu, w[3] & 0x7FFF7FFFu)];
+        __stcs(reinterpret_cast<uint2*>(vr + half * 8u),
+               make_uint2(__byte_perm(w[0], w[1], e0 >> 16), __byte_perm(w[2], w[3], e1 >> 16)));
+        mbyte = (e0 & 0xFu) | ((e1 & 0xFu) << 4);
+        if (COUNT)
+          lost += __popc(Group16::nonzero(w[0], w[1]) & ~(e0 >> 4) & 0xFu) +
+                  __popc(Group16::nonzero(w[2], w[3]) & ~(e1 >> 4) & 0xFu);
       }
-      uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, mbyte, 1);
-      if ((threadIdx.x & 1) == 0 && half < halves_pad)
-        *reinterpret_cast<uint16_t*>(meta + meta_offset<2>(layout, row, half >> 1, K, KB)) =
-            (uint16_t)(mbyte | (other << 8));
+      const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, mbyte, 1);
+      if ((threadIdx.x & 1) == 0 && (FULL || half < halves_pad))
+        *reinterpret_cast<uint16_t*>(mr + moff[u]) = (uint16_t)(mbyte | (other << 8));
     }
   }
   count_dropped<COUNT>(lost, dropped);
@@ -253,46 +264,56 @@ __global__ void __launch_bounds__(kThreads, 4) compress16_kernel(const uint8_t* 
 
 // int8.  Work unit: one chunk of 16 columns (four groups) = one 16-byte load, 8 bytes of values and
 // 16 bits of metadata out.
-template <int UNROLL, bool COUNT>
+template <int UNROLL, bool COUNT, bool HW, bool FULL>
 __global__ void __launch_bounds__(kThreads, 4) compress8_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
                                                              uint8_t* __restrict__ vals, int64_t row_bytes_v,
-                                                             uint8_t* __restrict__ meta, int layout, int64_t M,
-                                                             int64_t K, int64_t rows_pad, int64_t chunks_pad,
+                                                             uint8_t* __restrict__ meta, int64_t M, int64_t K,
+                                                             int64_t rows_pad, int64_t chunks_pad,
                                                              unsigned long long* dropped) {
   __shared__ uint32_t table[64];
   build_selection_table(table);
-  const int64_t chunks = K >> 4, KB = chunks_pad >> 3;
-  const int64_t c0 = (int64_t)blockIdx.x * UNROLL * blockDim.x + threadIdx.x;
+  const uint32_t chunks = (uint32_t)(K >> 4), cpad = (uint32_t)chunks_pad, KB = (uint32_t)(chunks_pad >> 3);
+  const uint32_t c0 = blockIdx.x * UNROLL * blockDim.x + threadIdx.x;
+  uint32_t moff[UNROLL];
+#pragma unroll
+  for (int u = 0; u < UNROLL; ++u) {
+    const uint32_t chunk = c0 + u * blockDim.x;
+    moff[u] = HW ? (chunk >> 3) * 2048u + 2u * (chunk & 7u) : 2u * chunk;
+  }
   uint32_t lost = 0;
   for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows_pad;
        row += (int64_t)gridDim.y * blockDim.y) {
+    const uint8_t* xr = x + row * row_bytes_x;
+    uint8_t* vr = vals + row * row_bytes_v;
+    uint8_t* mr = HW ? meta + (row >> 7) * ((int64_t)KB * 2048) + 16u * ((uint32_t)row & 127u) : meta + row * (K >> 3);
+    const bool row_live = FULL || row < M;
     uint4 in[UNROLL];
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
-      int64_t chunk = c0 + (int64_t)u * blockDim.x;
-      if (row < M && chunk < chunks) in[u] = ld_stream(x + row * row_bytes_x + chunk * 16);
+      const uint32_t chunk = c0 + u * blockDim.x;
+      if (row_live && (FULL || chunk < chunks)) in[u] = ld_stream(xr + chunk * 16u);
     }
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
-      int64_t chunk = c0 + (int64_t)u * blockDim.x;
-      if (chunk >= chunks_pad) continue;
+      const uint32_t chunk = c0 + u * blockDim.x;
+      if (!FULL && chunk >= cpad) continue;
       uint32_t mbits = 0x4444u;
-      if (row < M && chunk < chunks) {
-        uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
+      if (row_live && (FULL || chunk < chunks)) {
+        const uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
         uint32_t out[2] = {0, 0};
         mbits = 0;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-          uint32_t a = __vabs4(w[g]);  // -128 -> 0x80 = 128, no saturation
-          uint32_t e = table[selection_index(__byte_perm(a, 0, 0x4140), __byte_perm(a, 0, 0x4342))];
-          uint32_t pair = __byte_perm(w[g], 0, ((e >> 8) & 0xFFu) | 0x4400u);
+          const uint32_t a = __vabs4(w[g]);  // -128 -> 0x80 = 128, no saturation
+          const uint32_t e = table[selection_index(__byte_perm(a, 0, 0x4140), __byte_perm(a, 0, 0x4342))];
+          const uint32_t pair = __byte_perm(w[g], 0, ((e >> 8) & 0xFFu) | 0x4400u);
           out[g >> 1] |= pair << (16 * (g & 1));
           mbits |= (e & 0xFu) << (4 * g);
           if (COUNT) lost += __popc(Group8::nonzero(w[g]) & ~(e >> 4) & 0xFu);
         }
-        __stcs(reinterpret_cast<uint2*>(vals + row * row_bytes_v + chunk * 8), make_uint2(out[0], out[1]));
+        __stcs(reinterpret_cast<uint2*>(vr + chunk * 8u), make_uint2(out[0], out[1]));
       }
-      *reinterpret_cast<uint16_t*>(meta + meta_offset<1>(layout, row, chunk, K, KB)) = (uint16_t)mbits;
+      *reinterpret_cast<uint16_t*>(mr + moff[u]) = (uint16_t)mbits;
     }
   }
   count_dropped<COUNT>(lost, dropped);
@@ -511,20 +532,41 @@ extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const v
     uint8_t *vs = (uint8_t*)vals, *ms = (uint8_t*)meta;
     if (es == 2) {
       RowLaunch L(chunks_pad * 2, rows_pad, UNROLL);
-      if (dropped)
-        compress16_kernel<UNROLL, true><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, (int)l, M, K, rows_pad,
-                                                                   chunks_pad, dropped);
-      else
-        compress16_kernel<UNROLL, false><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, (int)l, M, K, rows_pad,
-                                                                    chunks_pad, dropped);
+      const bool full = rows_pad == M && k_pad == K &&
+                        (chunks_pad * 2) % ((int64_t)L.block.x * UNROLL) == 0;
+      const int variant = (dropped ? 4 : 0) | (hw ? 2 : 0) | (full ? 1 : 0);
+#define SP24_C16(COUNT, HW, FULL)                                                                          \
+  compress16_kernel<UNROLL, COUNT, HW, FULL><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, M, K, \
+                                                                        rows_pad, chunks_pad, dropped)
+      switch (variant) {
+        case 0: SP24_C16(false, false, false); break;
+        case 1: SP24_C16(false, false, true); break;
+        case 2: SP24_C16(false, true, false); break;
+        case 3: SP24_C16(false, true, true); break;
+        case 4: SP24_C16(true, false, false); break;
+        case 5: SP24_C16(true, false, true); break;
+        case 6: SP24_C16(true, true, false); break;
+        default: SP24_C16(true, true, true); break;
+      }
+#undef SP24_C16
     } else {
       RowLaunch L(chunks_pad, rows_pad, UNROLL);
-      if (dropped)
-        compress8_kernel<UNROLL, true><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, (int)l, M, K, rows_pad,
-                                                                  chunks_pad, dropped);
-      else
-        compress8_kernel<UNROLL, false><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, (int)l, M, K, rows_pad,
-                                                                   chunks_pad, dropped);
+      const bool full = rows_pad == M && k_pad == K && chunks_pad % ((int64_t)L.block.x * UNROLL) == 0;
+      const int variant = (dropped ? 4 : 0) | (hw ? 2 : 0) | (full ? 1 : 0);
+#define SP24_C8(COUNT, HW, FULL)                                                                          \
+  compress8_kernel<UNROLL, COUNT, HW, FULL><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, M, K, \
+                                                                       rows_pad, chunks_pad, dropped)
+      switch (variant) {
+        case 0: SP24_C8(false, false, false); break;
+        case 1: SP24_C8(false, false, true); break;
+        case 2: SP24_C8(false, true, false); break;
+        case 3: SP24_C8(false, true, true); break;
+        case 4: SP24_C8(true, false, false); break;
+        case 5: SP24_C8(true, false, true); break;
+        case 6: SP24_C8(true, true, false); break;
+        default: SP24_C8(true, true, true); break;
+      }
+#undef SP24_C8
     }
   } else {
     int64_t bytes_pad = k_pad / 8, total = rows_pad * bytes_pad;

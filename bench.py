@@ -304,6 +304,9 @@ def run_ours(args, cfg):
             ts = []
             for _ in range(reps):
                 flush.zero_()
+                # keep the GPU busy while the host enqueues, so that launch latency of these short
+                # kernels is not part of the interval between the two events
+                torch.cuda._sleep(400000)
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(stream)
                 fn()

@@ -37,7 +37,7 @@ namespace {
 constexpr int kBlockM = 128;              // rows of A per CTA and m-block (tensor-memory lanes)
 constexpr int kAtomBytes = 128;           // bytes per row of one swizzle-128B operand atom
 constexpr int kNumThreads = 192;          // 6 warps
-constexpr uint64_t kWaitTimeoutNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
+constexpr long long kWaitTimeoutCycles = 2000ll * 1000ll * 1000ll;  // per wait: 1-2 s of SM clock
 constexpr uint32_t kTmemCols = 512;
 
 struct GemmParams {
@@ -97,14 +97,17 @@ static_assert(sizeof(Shared) <= 512, "barrier block");
 
 __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, Shared* sh, uint32_t* status,
                                              uint32_t code) {
-  if (ptx::mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = ptx::globaltimer_ns();
+  // fast path: poll a while before any bookkeeping; try_wait itself suspends the thread briefly
+#pragma unroll 1
+  for (int i = 0; i < 64; ++i)
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
   uint32_t spins = 0;
   while (true) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
-    if ((++spins & 63u) == 0) {
+    if ((++spins & 255u) == 0) {
       if (sh->abort) return false;
-      if (ptx::globaltimer_ns() - t0 > kWaitTimeoutNs) {
+      if (clock64() - t0 > kWaitTimeoutCycles) {
         sh->abort = 1;
         atomicCAS(status, 0u, code);
         return false;
@@ -588,7 +591,18 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
     map_c = map_d;
   }
   auto kernel = gemm_kernel<KIND, SPARSE, BLOCK_N, CTAS, MBLK>;
-  SP24_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+  {
+    // the shared-memory opt-in is per kernel and device: once is enough
+    static std::mutex mu;
+    static bool done[64] = {};
+    int dev = 0;
+    SP24_CUDA_CHECK(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(mu);
+    if (dev < 0 || dev >= 64 || !done[dev]) {
+      SP24_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+      if (dev >= 0 && dev < 64) done[dev] = true;
+    }
+  }
   const int tiles = p.m_tiles * p.n_tiles;
   int clusters = sm_count() / CTAS;
   if (clusters > tiles) clusters = tiles;

@@ -125,7 +125,8 @@ sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals
  *   lda:     leading dimension of the A-side value array: of vals (M x K/2) when
  *            a_is_dense == 0, of the dense M x K matrix when a_is_dense == 1.
  *   order_b: SP24_COL_MAJOR = K contiguous (B stored as N rows of K values: the
- *            [tokens, hidden] activation layout), the only order built so far.
+ *            [tokens, hidden] activation layout; ldb >= K), the faster order, or
+ *            SP24_ROW_MAJOR = N contiguous (the K x N matrix stored row by row; ldb >= N).
  *   order_c / order_d: SP24_ROW_MAJOR (N contiguous).
  *   a_is_dense: 0 = 2:4 compressed A with TCGEN05 metadata (the sparse tensor-core path);
  *            1 = the dense variant on the same pipeline (`A` is M x K dense, `meta` unused).

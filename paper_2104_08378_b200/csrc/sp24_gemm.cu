@@ -55,7 +55,7 @@ struct GemmParams {
   int32_t band;       // m-tiles per band of the tile sweep
 };
 
-template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK>
+template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK, bool B_MN>
 struct Cfg {
   // 128-byte atoms per stage: sparse A is half as wide as B; the dense variant with two
   // m-blocks takes one atom per operand so that four stages still fit
@@ -64,7 +64,13 @@ struct Cfg {
   static constexpr int kBRows = BLOCK_N / CTAS;                    // B rows (N) this CTA loads
   static constexpr int kABlockBytes = kABoxes * kBlockM * kAtomBytes;  // one m-block
   static constexpr int kABytes = MBLK * kABlockBytes;
-  static constexpr int kBBytes = kBBoxes * kBRows * kAtomBytes;
+  static constexpr int kKPerStage = (KIND == 0 ? 64 : 128) * kBBoxes;  // logical K per stage
+  // B with N contiguous (MN-major operand): 128-byte chunks along N, each kKPerStage k-rows of 128 bytes
+  static constexpr int kBChunkElems = KIND == 0 ? 64 : 128;
+  static constexpr int kBChunks = (kBRows + kBChunkElems - 1) / kBChunkElems;
+  static constexpr int kBChunkBytes = kKPerStage * kAtomBytes;
+  static constexpr int kBKStepBytes = (SPARSE ? 2 : 1) * (KIND == 0 ? 16 : 32) * kAtomBytes;  // k-rows of one MMA
+  static constexpr int kBBytes = B_MN ? kBChunks * kBChunkBytes : kBBoxes * kBRows * kAtomBytes;
   static constexpr int kEBlocks = SPARSE ? (KIND == 0 ? 1 : 2) : 0;  // 2048-byte metadata blocks per m-block and stage
   static constexpr int kEBlockBytes = kEBlocks * 2048;
   static constexpr int kEBytes = MBLK * kEBlockBytes;
@@ -78,7 +84,6 @@ struct Cfg {
   static constexpr int kAccStages = MBLK == 2 ? 1 : ((2 * BLOCK_N + (SPARSE ? 32 : 0) <= (int)kTmemCols) ? 2 : 1);
   static constexpr int kECol = kAccStages * MBLK * BLOCK_N;        // first metadata column in tensor memory
   static constexpr int kMmasPerStage = SPARSE ? 4 : 4 * kBBoxes;   // per m-block
-  static constexpr int kKPerStage = (KIND == 0 ? 64 : 128) * kBBoxes;  // logical K per stage
   static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
   static_assert(kStages >= 2, "need at least two stages");
   static_assert(BLOCK_N % 32 == 0, "the epilogue moves 32-column boxes");
@@ -127,16 +132,17 @@ __device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int
 }
 
 template <int KIND>
-__device__ __forceinline__ uint32_t make_idesc(bool sparse, int a_fmt, int m, int n) {
+__device__ __forceinline__ uint32_t make_idesc(bool sparse, bool b_mn_major, int a_fmt, int m, int n) {
   uint32_t d = 0;
   d |= (sparse ? 1u : 0u) << 2;
   d |= (KIND == 0 ? 1u : 2u) << 4;                 // accumulator: fp32 / int32
   uint32_t fmt = KIND == 0 ? (uint32_t)a_fmt : 1u;  // f16 = 0, bf16 = 1; int8: 1 = signed
   d |= fmt << 7;
   d |= fmt << 10;
+  d |= (b_mn_major ? 1u : 0u) << 16;               // A is always K-major
   d |= (uint32_t)(n >> 3) << 17;
   d |= (uint32_t)(m >> 4) << 24;
-  return d;                                        // both operands K-major, no negate, no saturate
+  return d;                                        // no negate, no saturate
 }
 
 // ---- epilogue helpers ----------------------------------------------------------------------------
@@ -207,12 +213,12 @@ __device__ __forceinline__ void convert_row(const uint32_t (&r)[32], uint8_t* bu
   }
 }
 
-template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK>
+template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK, bool B_MN>
 __global__ void __launch_bounds__(kNumThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_e, const __grid_constant__ CUtensorMap map_c,
             const __grid_constant__ CUtensorMap map_d, const GemmParams p) {
-  using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS, MBLK>;
+  using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS, MBLK, B_MN>;
   extern __shared__ uint8_t smem_raw[];
   // Operand atoms need 1024-byte alignment for the 128-byte swizzle.
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -299,11 +305,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               else ptx::tma_load_2d_pair(se + j * C::kEBlockBytes, &map_e, full, 0, 0, y);
             }
           }
+          if (B_MN) {
+            // B stored N-contiguous: boxes of 128 bytes along N x all k-rows of the stage
 #pragma unroll
-          for (int i = 0; i < C::kBBoxes; ++i) {
-            int x = (kb * C::kBBoxes + i) * box_elems;
-            if (CTAS == 1) ptx::tma_load_2d(sb + i * C::kBRows * kAtomBytes, &map_b, full, x, col0);
-            else ptx::tma_load_2d_pair(sb + i * C::kBRows * kAtomBytes, &map_b, full, 0, x, col0);
+            for (int c = 0; c < C::kBChunks; ++c) {
+              int x = col0 + c * C::kBChunkElems, y = kb * C::kKPerStage;
+              if (CTAS == 1) ptx::tma_load_2d(sb + c * C::kBChunkBytes, &map_b, full, x, y);
+              else ptx::tma_load_2d_pair(sb + c * C::kBChunkBytes, &map_b, full, 0, x, y);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < C::kBBoxes; ++i) {
+              int x = (kb * C::kBBoxes + i) * box_elems;
+              if (CTAS == 1) ptx::tma_load_2d(sb + i * C::kBRows * kAtomBytes, &map_b, full, x, col0);
+              else ptx::tma_load_2d_pair(sb + i * C::kBRows * kAtomBytes, &map_b, full, 0, x, col0);
+            }
           }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
@@ -321,7 +337,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int n_eff = min(BLOCK_N, (int)(p.N - (int64_t)nt * BLOCK_N));
         const int live = min(MBLK, (int)((p.M - (int64_t)mt * MBLK * CTAS * kBlockM + CTAS * kBlockM - 1) /
                                          (CTAS * kBlockM)));
-        const uint32_t idesc = make_idesc<KIND>(SPARSE, p.a_fmt, kBlockM * CTAS, n_eff);
+        const uint32_t idesc = make_idesc<KIND>(SPARSE, B_MN, p.a_fmt, kBlockM * CTAS, n_eff);
         if (!bounded_wait(&sh->tmem_empty[acc], acc_phase ^ 1u, sh, p.status, 2u)) break;
         ptx::tc_fence_after();
         bool ok = true;
@@ -356,7 +372,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               if (SPARSE) {
                 // 32 bytes of compressed A and 64 bytes of B per instruction
                 uint64_t da = ptx::smem_desc(saj + k * 32, true, 1024);
-                uint64_t db = ptx::smem_desc(sb + (k >> 1) * C::kBRows * kAtomBytes + (k & 1) * 64, true, 1024);
+                uint64_t db = B_MN ? ptx::smem_desc(sb + k * C::kBKStepBytes, true, 1024, C::kBChunkBytes)
+                                   : ptx::smem_desc(sb + (k >> 1) * C::kBRows * kAtomBytes + (k & 1) * 64, true, 1024);
                 if (KIND == 0) {
                   // one 32-bit metadata column per instruction: even-aligned address + selector
                   ptx::mma_sparse<KIND, CTAS>(d_tmem, da, db, e_tmem + (k & ~1), idesc | (uint32_t)(k & 1), accumulate);
@@ -365,7 +382,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 }
               } else {
                 uint64_t da = ptx::smem_desc(saj + (k >> 2) * kBlockM * kAtomBytes + (k & 3) * 32, true, 1024);
-                uint64_t db = ptx::smem_desc(sb + (k >> 2) * C::kBRows * kAtomBytes + (k & 3) * 32, true, 1024);
+                uint64_t db = B_MN ? ptx::smem_desc(sb + k * C::kBKStepBytes, true, 1024, C::kBChunkBytes)
+                                   : ptx::smem_desc(sb + (k >> 2) * C::kBRows * kAtomBytes + (k & 3) * 32, true, 1024);
                 ptx::mma_dense<KIND, CTAS>(d_tmem, da, db, idesc, accumulate);
               }
             }
@@ -554,10 +572,10 @@ int sm_count() {
   return n;
 }
 
-template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK>
+template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK, bool B_MN>
 sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* A, const void* meta, const void* B,
                    cudaStream_t stream) {
-  using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS, MBLK>;
+  using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS, MBLK, B_MN>;
   GemmParams p = base;
   const int es = KIND == 0 ? 2 : 1;
   const int tile_m = kBlockM * CTAS * MBLK;
@@ -570,7 +588,8 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
   const uint64_t a_cols = SPARSE ? d->K / 2 : d->K;
   sp24_status st = make_map(&map_a, A, es, d->M, a_cols, d->lda * es, atom_elems, kBlockM, 128);
   if (st != SP24_OK) return st;
-  st = make_map(&map_b, B, es, d->N, d->K, d->ldb * es, atom_elems, C::kBRows, 128);
+  if (B_MN) st = make_map(&map_b, B, es, d->K, d->N, d->ldb * es, C::kBChunkElems, C::kKPerStage, 128);
+  else st = make_map(&map_b, B, es, d->N, d->K, d->ldb * es, atom_elems, C::kBRows, 128);
   if (st != SP24_OK) return st;
   if (SPARSE) {
     uint64_t meta_rows = (uint64_t)((d->M + 127) / 128) * p.meta_kb * 16;  // rows of 128 bytes
@@ -590,7 +609,7 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
   } else {
     map_c = map_d;
   }
-  auto kernel = gemm_kernel<KIND, SPARSE, BLOCK_N, CTAS, MBLK>;
+  auto kernel = gemm_kernel<KIND, SPARSE, BLOCK_N, CTAS, MBLK, B_MN>;
   {
     // the shared-memory opt-in is per kernel and device: once is enough
     static std::mutex mu;
@@ -644,8 +663,8 @@ static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, con
   SP24_RETURN_IF(d->M < 0 || d->N < 0 || d->K <= 0, SP24_ERR_SHAPE);
   SP24_RETURN_IF(d->M % mult || d->N % mult || d->K % mult, SP24_ERR_SHAPE);
   SP24_RETURN_IF(d->M > (int64_t(1) << 30) || d->N > (int64_t(1) << 30) || d->K > (int64_t(1) << 30), SP24_ERR_SHAPE);
-  SP24_RETURN_IF(d->order_b != SP24_COL_MAJOR || d->order_c != SP24_ROW_MAJOR || d->order_d != SP24_ROW_MAJOR,
-                 SP24_ERR_UNSUPPORTED);
+  SP24_RETURN_IF(d->order_b != SP24_COL_MAJOR && d->order_b != SP24_ROW_MAJOR, SP24_ERR_UNSUPPORTED);
+  SP24_RETURN_IF(d->order_c != SP24_ROW_MAJOR || d->order_d != SP24_ROW_MAJOR, SP24_ERR_UNSUPPORTED);
   if (fp) {
     falpha = *static_cast<const float*>(alpha);
     fbeta = *static_cast<const float*>(beta);
@@ -662,7 +681,9 @@ static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, con
   SP24_RETURN_IF(ws == nullptr || ws_bytes < 256 || !aligned16(ws), SP24_ERR_WORKSPACE);
   const int es = elem_bytes(d->ab_type), cs = elem_bytes(d->cd_type);
   const int64_t a_cols = d->a_is_dense ? d->K : d->K / 2;
-  SP24_RETURN_IF(d->lda < a_cols || d->ldb < d->K || d->ldd < d->N || (has_c && d->ldc < d->N), SP24_ERR_STRIDE);
+  SP24_RETURN_IF(d->lda < a_cols || d->ldb < (d->order_b == SP24_COL_MAJOR ? d->K : d->N) || d->ldd < d->N ||
+                     (has_c && d->ldc < d->N),
+                 SP24_ERR_STRIDE);
   SP24_RETURN_IF((d->lda * es) % 16 || (d->ldb * es) % 16 || (d->ldd * cs) % 16 || (has_c && (d->ldc * cs) % 16),
                  SP24_ERR_STRIDE);
   SP24_RETURN_IF(!aligned16(A) || !aligned16(B) || !aligned16(D) || (has_c && !aligned16(C)) ||
@@ -711,17 +732,24 @@ extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, con
     int b = atoi(env);
     if (b > 0) p.band = b;
   }
-#define SP24_DISPATCH(CT, BN, MB)                                                                            \
-  if (ctas == CT && block_n == BN && mblk == MB) {                                                           \
-    if (!i8) return sparse ? launch<0, true, BN, CT, MB>(d, p, A, meta, B, s) : launch<0, false, BN, CT, MB>(d, p, A, meta, B, s); \
-    return sparse ? launch<1, true, BN, CT, MB>(d, p, A, meta, B, s) : launch<1, false, BN, CT, MB>(d, p, A, meta, B, s);          \
-  }
+  const bool b_mn = d->order_b == SP24_ROW_MAJOR;  // B stored N-contiguous
+#define SP24_LAUNCH(K_, BN, CT, MB, MN)                                                               \
+  (sparse ? launch<K_, true, BN, CT, MB, MN>(d, p, A, meta, B, s) : launch<K_, false, BN, CT, MB, MN>(d, p, A, meta, B, s))
+#define SP24_DISPATCH(CT, BN, MB)                                                                     \
+  if (ctas == CT && block_n == BN && mblk == MB && !b_mn) return i8 ? SP24_LAUNCH(1, BN, CT, MB, false) : SP24_LAUNCH(0, BN, CT, MB, false);
+#define SP24_DISPATCH_MN(CT, BN, MB)                                                                  \
+  if (ctas == CT && block_n == BN && mblk == MB && b_mn) return i8 ? SP24_LAUNCH(1, BN, CT, MB, true) : SP24_LAUNCH(0, BN, CT, MB, true);
   SP24_DISPATCH(1, 128, 1)
   SP24_DISPATCH(2, 224, 1)
   SP24_DISPATCH(2, 224, 2)
   SP24_DISPATCH(2, 192, 2)
   SP24_DISPATCH(2, 256, 1)
+  SP24_DISPATCH_MN(1, 128, 1)
+  SP24_DISPATCH_MN(2, 224, 1)
+  SP24_DISPATCH_MN(2, 224, 2)
 #undef SP24_DISPATCH
+#undef SP24_DISPATCH_MN
+#undef SP24_LAUNCH
   return SP24_ERR_UNSUPPORTED;
 }
 

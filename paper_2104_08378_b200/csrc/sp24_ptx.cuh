@@ -156,12 +156,17 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
 }
 
 // ---- descriptors ---------------------------------------------------------------------------------
-// Shared-memory matrix descriptor, K-major operand.  `swizzle128`: rows of 128 bytes, 8-row
-// groups 1024 bytes apart, 128-byte swizzle (what the TMA loads write).  Otherwise no swizzle:
-// 8 x 16-byte core matrices `sbo` bytes apart along rows.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t smem_addr, bool swizzle128, uint32_t sbo_bytes) {
+// Shared-memory matrix descriptor for a 128-byte-swizzled operand (what the TMA loads write) or,
+// with `swizzle128` false, for 8 x 16-byte core matrices without swizzle.
+//   K-major operand:  rows of 128 bytes along K, 8-row groups `sbo_bytes` (1024) apart; lbo unused.
+//   MN-major operand: rows of 128 bytes along M/N (64 16-bit or 128 8-bit elements), consecutive k
+//                     128 bytes apart, groups of 8 k `sbo_bytes` (1024) apart, 128-byte chunks along
+//                     M/N `lbo_bytes` apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t smem_addr, bool swizzle128, uint32_t sbo_bytes,
+                                              uint32_t lbo_bytes = 0) {
   uint64_t d = 0;
   d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
   d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
   d |= (uint64_t)1 << 46;  // descriptor version for sm_100
   if (swizzle128) d |= (uint64_t)2 << 61;

@@ -118,6 +118,35 @@ def test_alpha_beta_with_c(sp):
     run_case(sp, cfg, cd="f32", alpha=1.0, beta=1.0)
 
 
+@pytest.mark.parametrize("dense", [False, True])
+@pytest.mark.parametrize("case", [("bf16", 128, 128, 128), ("f16", 144, 272, 400), ("bf16", 512, 672, 1024),
+                                  ("bf16", 1024, 9472, 256), ("i8", 160, 288, 416), ("i8", 512, 1344, 1024)])
+def test_b_stored_n_contiguous(sp, dense, case):
+    """order_b = ROW_MAJOR: the K x N matrix stored row by row (MN-major tensor-core operand)."""
+    ab, M, N, K = case
+    base = inputs.CONFIGS["int8_linear" if ab == "i8" else ("tiny_f16" if ab == "f16" else "bert_ffn_bf16")]
+    cfg = inputs.scaled(base, M=M, N=N, K=K)
+    A, Bt = inputs.gen_A(cfg), inputs.gen_Bt(cfg)
+    vals_ref, meta_ref, _ = oracle.compress(A, ab)
+    Ad = to_device(A, ab)
+    Bkn = to_device(np.ascontiguousarray(Bt.T), ab)          # [K, N], N contiguous
+    cd = "i32" if ab == "i8" else "f32"
+    if dense:
+        D = sp.gemm(sp.prune(Ad), None, Bkn, cd=cd, a_is_dense=True, b_row_major=True)
+    else:
+        vals, meta, _ = sp.compress(Ad)
+        D = sp.gemm(vals, meta, Bkn, cd=cd, b_row_major=True)
+    torch.cuda.synchronize()
+    assert sp.gemm_status(device=D.device) == 0
+    rows, cols = (0, min(M, 256)), (max(0, N - 320), N)      # a window keeps the oracle quick
+    ref = oracle.gemm_sparse(vals_ref, meta_ref, Bt, ab, rows=rows, cols=cols)
+    got = to_host_f64(D[rows[0]:rows[1], cols[0]:cols[1]])
+    if ab == "i8":
+        assert np.array_equal(got, ref)
+    else:
+        check_fp(got, ref, oracle.gemm_abs(vals_ref, meta_ref, Bt, ab, rows=rows, cols=cols))
+
+
 def test_identity_b_returns_decompressed_a(sp):
     """B = I: the sparse GEMM must reproduce prune(A) exactly (every selected index is exercised)."""
     for ab, K in (("f16", 256), ("bf16", 384), ("i8", 512)):

@@ -127,7 +127,9 @@ sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals
  *   order_b: SP24_COL_MAJOR = K contiguous (B stored as N rows of K values: the
  *            [tokens, hidden] activation layout; ldb >= K), the faster order, or
  *            SP24_ROW_MAJOR = N contiguous (the K x N matrix stored row by row; ldb >= N).
- *   order_c / order_d: SP24_ROW_MAJOR (N contiguous).
+ *   order_c / order_d: SP24_ROW_MAJOR (N contiguous; ldc, ldd >= N) or SP24_COL_MAJOR
+ *            (M contiguous, the [tokens, out_features] layout; ldc, ldd >= M).  When C is
+ *            used (beta != 0) it must have the same order as D.
  *   a_is_dense: 0 = 2:4 compressed A with TCGEN05 metadata (the sparse tensor-core path);
  *            1 = the dense variant on the same pipeline (`A` is M x K dense, `meta` unused).
  * All leading dimensions are in elements and, in bytes, multiples of 16. */

@@ -156,9 +156,10 @@ def decompress(vals: torch.Tensor, meta: torch.Tensor, layout: int = META_TCGEN0
 
 
 def make_desc(ab: str, cd: str, M: int, N: int, K: int, lda: int, ldb: int, ldc: int, ldd: int,
-              a_is_dense: bool = False, b_row_major: bool = False) -> GemmDesc:
+              a_is_dense: bool = False, b_row_major: bool = False, cd_col_major: bool = False) -> GemmDesc:
+    cd_order = COL_MAJOR if cd_col_major else ROW_MAJOR
     return GemmDesc(DTYPE_CODE[ab], DTYPE_CODE[cd], M, N, K, lda, ldb, ldc, ldd,
-                    ROW_MAJOR if b_row_major else COL_MAJOR, ROW_MAJOR, ROW_MAJOR, 1 if a_is_dense else 0)
+                    ROW_MAJOR if b_row_major else COL_MAJOR, cd_order, cd_order, 1 if a_is_dense else 0)
 
 
 def _scalar(ab: str, v):
@@ -178,9 +179,10 @@ def workspace(device) -> torch.Tensor:
 def gemm(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor, *, alpha=1.0, beta=0.0,
          C: torch.Tensor | None = None, out: torch.Tensor | None = None, cd: str | None = None,
          ab: str | None = None, a_is_dense: bool = False, ws: torch.Tensor | None = None,
-         b_row_major: bool = False) -> torch.Tensor:
+         b_row_major: bool = False, cd_col_major: bool = False) -> torch.Tensor:
     """sp24_gemm.  A: vals [M, K/2] (or dense [M, K]); Bt: [N, K] (K contiguous), or with
-    b_row_major=True the K x N matrix itself, [K, N] (N contiguous); C/D: [M, N]."""
+    b_row_major=True the K x N matrix itself, [K, N] (N contiguous); C/D: [M, N], or with
+    cd_col_major=True their transposes [N, M] (M contiguous)."""
     ab = _dtype_of(A, ab)
     M = A.shape[0]
     K = A.shape[1] if a_is_dense else 2 * A.shape[1]
@@ -188,10 +190,11 @@ def gemm(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor, *, alpha=
     assert (Bt.shape[0] if b_row_major else Bt.shape[1]) == K
     cd = cd or ("i32" if ab == "i8" else ab)
     if out is None:
-        out = torch.empty((M, N), dtype=TORCH_DTYPE[cd], device=A.device)
+        out = torch.empty((N, M) if cd_col_major else (M, N), dtype=TORCH_DTYPE[cd], device=A.device)
     ws = ws if ws is not None else workspace(A.device)
-    desc = make_desc(ab, cd, M, N, K, A.stride(0), Bt.stride(0), C.stride(0) if C is not None else N,
-                     out.stride(0), a_is_dense, b_row_major)
+    desc = make_desc(ab, cd, M, N, K, A.stride(0), Bt.stride(0),
+                     C.stride(0) if C is not None else (M if cd_col_major else N), out.stride(0), a_is_dense,
+                     b_row_major, cd_col_major)
     a, b = _scalar(ab, alpha), _scalar(ab, beta)
     _check(lib.sp24_gemm(ctypes.byref(desc), ctypes.byref(a), _ptr(A), _ptr(meta), _ptr(Bt),
                          ctypes.byref(b), _ptr(C), _ptr(out), _ptr(ws), ws.numel(), _stream()), "sp24_gemm")

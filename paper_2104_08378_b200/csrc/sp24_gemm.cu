@@ -53,6 +53,7 @@ struct GemmParams {
   int32_t cd_type;    // sp24_dtype of C / D
   int32_t has_c;
   int32_t band;       // m-tiles per band of the tile sweep
+  int32_t cd_col_major;  // C and D stored M-contiguous (the [tokens, out_features] layout)
 };
 
 template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK, bool B_MN>
@@ -209,6 +210,39 @@ __device__ __forceinline__ void convert_row(const uint32_t (&r)[32], uint8_t* bu
         }
       }
       *u = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+    }
+  }
+}
+
+// Column-major C / D: the staging buffer holds the box transposed (32 rows of n, m contiguous), so
+// this thread's 32 values go to 32 different rows, one element each.
+template <int KIND>
+__device__ __forceinline__ void convert_row_transposed(const uint32_t (&r)[32], uint8_t* buf, int lane,
+                                                       const GemmParams& p) {
+  const bool wide = KIND == 1 || p.cd_type == SP24_F32;
+#pragma unroll
+  for (int n = 0; n < 32; ++n) {
+    if (wide) {
+      uint32_t* u = reinterpret_cast<uint32_t*>(buf + n * 128 + ((((lane >> 2) ^ (n & 7))) << 4) + (lane & 3) * 4);
+      if (KIND == 1) {
+        *u = r[n] + (p.has_c ? *u : 0u);
+      } else {
+        float f = p.alpha * __uint_as_float(r[n]);
+        if (p.has_c) f += p.beta * __uint_as_float(*u);
+        *u = __float_as_uint(f);
+      }
+    } else {
+      uint16_t* u = reinterpret_cast<uint16_t*>(buf + n * 64 + ((((lane >> 3) ^ ((n >> 1) & 3))) << 4) + (lane & 7) * 2);
+      float f = p.alpha * __uint_as_float(r[n]);
+      if (p.cd_type == SP24_BF16) {
+        if (p.has_c) f += p.beta * __bfloat162float(*reinterpret_cast<__nv_bfloat16*>(u));
+        __nv_bfloat16 o = __float2bfloat16_rn(f);
+        *u = *reinterpret_cast<uint16_t*>(&o);
+      } else {
+        if (p.has_c) f += p.beta * __half2float(*reinterpret_cast<__half*>(u));
+        __half o = __float2half_rn(f);
+        *u = *reinterpret_cast<uint16_t*>(&o);
+      }
     }
   }
 }
@@ -436,7 +470,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (live_box) {
           const int b = pf_seq % nbuf;
           ptx::mbar_expect_tx(&sh->c_full[q][b], (uint32_t)buf_bytes);
-          ptx::tma_load_2d(my_bufs + b * buf_bytes, &map_c, &sh->c_full[q][b], col0, row0);
+          ptx::tma_load_2d(my_bufs + b * buf_bytes, &map_c, &sh->c_full[q][b], p.cd_col_major ? row0 : col0,
+                           p.cd_col_major ? col0 : row0);
           ++pf_seq;
           return;
         }
@@ -455,7 +490,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         for (uint32_t spin = 0; sh->c_hint_tiles < tiles_seen && spin < (1u << 20) && !sh->abort; ++spin) __nanosleep(128);
         for (int it = 0; it < kIters; ++it) {
           int row0, col0;
-          if (box_of(t, it, row0, col0)) ptx::tma_prefetch_2d(&map_c, col0, row0);
+          if (box_of(t, it, row0, col0))
+            ptx::tma_prefetch_2d(&map_c, p.cd_col_major ? row0 : col0, p.cd_col_major ? col0 : row0);
         }
       }
       if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u)) break;
@@ -479,11 +515,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int b = seq % nbuf;
         uint8_t* buf = my_bufs + b * buf_bytes;
         if (p.has_c && !bounded_wait(&sh->c_full[q][b], (seq / nbuf) & 1u, sh, p.status, 5u)) { ok = false; break; }
-        convert_row<KIND>(r, buf, lane, p);
+        if (p.cd_col_major) convert_row_transposed<KIND>(r, buf, lane, p);
+        else convert_row<KIND>(r, buf, lane, p);
         ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          ptx::tma_store_2d(&map_d, buf, col0, row0);
+          ptx::tma_store_2d(&map_d, buf, p.cd_col_major ? row0 : col0, p.cd_col_major ? col0 : row0);
           ptx::bulk_commit_group();
           // the buffer claimed next is free once the store that used it last has read it
           if (pending_ok >= 3) ptx::bulk_wait_group_read<3>();
@@ -601,10 +638,11 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
   // C and D move in 32 x 32 boxes whose rows are 64 bytes (2-byte types) or 128 bytes (4-byte types)
   CUtensorMap map_c, map_d;
   const int cs = elem_bytes(d->cd_type);
-  st = make_map(&map_d, p.D, cs, d->M, d->N, d->ldd * cs, 32, 32, 32 * cs);
+  const uint64_t cd_rows = p.cd_col_major ? d->N : d->M, cd_cols = p.cd_col_major ? d->M : d->N;
+  st = make_map(&map_d, p.D, cs, cd_rows, cd_cols, d->ldd * cs, 32, 32, 32 * cs);
   if (st != SP24_OK) return st;
   if (p.has_c) {
-    st = make_map(&map_c, p.C, cs, d->M, d->N, d->ldc * cs, 32, 32, 32 * cs);
+    st = make_map(&map_c, p.C, cs, cd_rows, cd_cols, d->ldc * cs, 32, 32, 32 * cs);
     if (st != SP24_OK) return st;
   } else {
     map_c = map_d;
@@ -664,7 +702,7 @@ static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, con
   SP24_RETURN_IF(d->M % mult || d->N % mult || d->K % mult, SP24_ERR_SHAPE);
   SP24_RETURN_IF(d->M > (int64_t(1) << 30) || d->N > (int64_t(1) << 30) || d->K > (int64_t(1) << 30), SP24_ERR_SHAPE);
   SP24_RETURN_IF(d->order_b != SP24_COL_MAJOR && d->order_b != SP24_ROW_MAJOR, SP24_ERR_UNSUPPORTED);
-  SP24_RETURN_IF(d->order_c != SP24_ROW_MAJOR || d->order_d != SP24_ROW_MAJOR, SP24_ERR_UNSUPPORTED);
+  SP24_RETURN_IF(d->order_d != SP24_ROW_MAJOR && d->order_d != SP24_COL_MAJOR, SP24_ERR_UNSUPPORTED);
   if (fp) {
     falpha = *static_cast<const float*>(alpha);
     fbeta = *static_cast<const float*>(beta);
@@ -675,14 +713,17 @@ static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, con
     fbeta = (float)ib;
   }
   has_c = fbeta != 0.f;
+  // C is converted in place into D inside the epilogue's staging buffer: same order for both
+  SP24_RETURN_IF(has_c && d->order_c != d->order_d, SP24_ERR_UNSUPPORTED);
   if (d->M == 0 || d->N == 0) return SP24_OK;
   SP24_RETURN_IF(A == nullptr || B == nullptr || D == nullptr || (has_c && C == nullptr), SP24_ERR_NULL);
   SP24_RETURN_IF(!d->a_is_dense && meta == nullptr, SP24_ERR_NULL);
   SP24_RETURN_IF(ws == nullptr || ws_bytes < 256 || !aligned16(ws), SP24_ERR_WORKSPACE);
   const int es = elem_bytes(d->ab_type), cs = elem_bytes(d->cd_type);
   const int64_t a_cols = d->a_is_dense ? d->K : d->K / 2;
-  SP24_RETURN_IF(d->lda < a_cols || d->ldb < (d->order_b == SP24_COL_MAJOR ? d->K : d->N) || d->ldd < d->N ||
-                     (has_c && d->ldc < d->N),
+  const int64_t cd_width = d->order_d == SP24_COL_MAJOR ? d->M : d->N;
+  SP24_RETURN_IF(d->lda < a_cols || d->ldb < (d->order_b == SP24_COL_MAJOR ? d->K : d->N) || d->ldd < cd_width ||
+                     (has_c && d->ldc < cd_width),
                  SP24_ERR_STRIDE);
   SP24_RETURN_IF((d->lda * es) % 16 || (d->ldb * es) % 16 || (d->ldd * cs) % 16 || (has_c && (d->ldc * cs) % 16),
                  SP24_ERR_STRIDE);
@@ -712,6 +753,7 @@ extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, con
   p.a_fmt = d->ab_type == SP24_BF16 ? 1 : 0;
   p.cd_type = (int)d->cd_type;
   p.has_c = has_c ? 1 : 0;
+  p.cd_col_major = d->order_d == SP24_COL_MAJOR ? 1 : 0;
   const bool sparse = !d->a_is_dense;
   const bool i8 = d->ab_type == SP24_I8;
   // Tile choice.  Large problems (at least six waves of tiles): a pair of CTAs with two m-blocks

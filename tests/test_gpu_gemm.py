@@ -147,6 +147,73 @@ def test_b_stored_n_contiguous(sp, dense, case):
         check_fp(got, ref, oracle.gemm_abs(vals_ref, meta_ref, Bt, ab, rows=rows, cols=cols))
 
 
+@pytest.mark.parametrize("case", [("bf16", "bf16", 272, 464, 528, 1.0), ("f16", "f32", 128, 160, 256, -0.5),
+                                  ("i8", "i32", 288, 352, 512, 1), ("bf16", "bf16", 1024, 9472, 256, 0.0)])
+def test_c_and_d_stored_m_contiguous(sp, case):
+    """order_c = order_d = COL_MAJOR: D^T ([N, M], the [tokens, out_features] layout)."""
+    ab, cd, M, N, K, beta = case
+    base = inputs.CONFIGS["int8_linear" if ab == "i8" else "bert_ffn_bf16"]
+    cfg = inputs.scaled(base, M=M, N=N, K=K)
+    if ab == "f16":
+        cfg = inputs.scaled(inputs.CONFIGS["tiny_f16"], M=M, N=N, K=K)
+    A, Bt = inputs.gen_A(cfg), inputs.gen_Bt(cfg)
+    vals_ref, meta_ref, _ = oracle.compress(A, ab)
+    Cm = Cd = None
+    if beta != 0:
+        if ab == "i8":
+            Cm = inputs._matrix(("int8",), "i8", 5, inputs.TENSOR_C, N, 0, M).astype(np.int32)
+        else:
+            Cm = inputs._matrix(("normal", 1.0), "bf16", 5, inputs.TENSOR_C, N, 0, M)
+            if cd == "f32":
+                Cm = np.ascontiguousarray(oracle.bits_to_float64(Cm, "bf16").astype(np.float32))
+        Cd = to_device(np.ascontiguousarray(Cm.T), cd)           # [N, M]
+    vals, meta, _ = sp.compress(to_device(A, ab))
+    Dt = sp.gemm(vals, meta, to_device(Bt, ab), alpha=1 if ab == "i8" else 2.0, beta=beta, C=Cd, cd=cd,
+                 cd_col_major=True)
+    torch.cuda.synchronize()
+    assert Dt.shape == (N, M)
+    alpha = 1 if ab == "i8" else 2.0
+    rows, cols = (0, min(M, 288)), (max(0, N - 352), N)
+    ref = oracle.gemm_sparse(vals_ref, meta_ref, Bt, ab, alpha, beta, Cm, cd if Cm is not None else None,
+                             rows=rows, cols=cols)
+    got = to_host_f64(Dt.t()[rows[0]:rows[1], cols[0]:cols[1]])
+    if ab == "i8":
+        assert np.array_equal(got, ref)
+    else:
+        scale = abs(alpha) * oracle.gemm_abs(vals_ref, meta_ref, Bt, ab, rows=rows, cols=cols)
+        beta_c = None
+        if Cm is not None:
+            csub = np.ascontiguousarray(Cm[rows[0]:rows[1], cols[0]:cols[1]])
+            beta_c = abs(beta) * np.abs(oracle.bits_to_float64(csub, cd) if cd != "f32" else csub)
+        check_fp(got, ref, scale, beta_c)
+
+
+def test_leading_dimensions_larger_than_the_matrices(sp):
+    """Every operand as a window of a wider allocation (lda, ldb, ldc, ldd > logical width)."""
+    cfg = inputs.scaled(inputs.CONFIGS["gpt3_ffn_bf16"], M=272, N=464, K=528)
+    M, N, K = cfg.M, cfg.N, cfg.K
+    A, Bt, Cm = inputs.gen_A(cfg), inputs.gen_Bt(cfg), inputs.gen_C(cfg)
+    vals_ref, meta_ref, _ = oracle.compress(A, "bf16")
+    vals_t, meta, _ = sp.compress(to_device(A, "bf16"))
+    pad = lambda t, extra: torch.nn.functional.pad(t.view(torch.int16), (0, extra)).view(t.dtype)  # noqa: E731
+    vals_w = pad(vals_t, 24)[:, :K // 2]                      # lda = K/2 + 24
+    Bt_w = pad(to_device(Bt, "bf16"), 40)[:, :K]              # ldb = K + 40
+    C_w = pad(to_device(Cm, "bf16"), 16)[:, :N]               # ldc = N + 16
+    D_full = torch.full((M, N + 48), 7.0, dtype=torch.bfloat16, device="cuda")
+    D_w = D_full[:, :N]                                       # ldd = N + 48
+    sp.gemm(vals_w, meta, Bt_w, alpha=1.0, beta=1.0, C=C_w, out=D_w)
+    torch.cuda.synchronize()
+    ref = oracle.gemm_sparse(vals_ref, meta_ref, Bt, "bf16", 1.0, 1.0, Cm, "bf16")
+    scale = oracle.gemm_abs(vals_ref, meta_ref, Bt, "bf16")
+    check_fp(to_host_f64(D_w), ref, scale, np.abs(oracle.bits_to_float64(Cm, "bf16")))
+    assert torch.all(D_full[:, N:] == 7.0)                    # nothing written past column N
+    # C aliasing D (in-place accumulate)
+    D2 = to_device(Cm, "bf16").clone()
+    sp.gemm(vals_t, meta, to_device(Bt, "bf16"), alpha=1.0, beta=1.0, C=D2, out=D2)
+    torch.cuda.synchronize()
+    check_fp(to_host_f64(D2), ref, scale, np.abs(oracle.bits_to_float64(Cm, "bf16")))
+
+
 def test_identity_b_returns_decompressed_a(sp):
     """B = I: the sparse GEMM must reproduce prune(A) exactly (every selected index is exercised)."""
     for ab, K in (("f16", 256), ("bf16", 384), ("i8", 512)):

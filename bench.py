@@ -339,6 +339,16 @@ def run_ours(args, cfg):
                             "dense_variant_ms": d_ms, "speedup_vs_dense_variant": d_ms / s_ms}
             if im2col_ms is not None:
                 others[name]["im2col_ms"] = im2col_ms
+            if oc.ab_type == "i8":
+                # the dequantising epilogue (per-row scales) with bf16 and int8 outputs
+                rs = torch.full((oc.M,), 1e-5, dtype=torch.float32, device=dev)
+                for out_t in ("bf16", "i8"):
+                    oQ = torch.empty((oc.M, oc.N), dtype=tdt[out_t], device=dev)
+                    q_ms = time_flushed(lambda: sp.gemm_i8_dequant(ovals, ometa, oB, rs, cd=out_t, out_scale=0.05,
+                                                                   out=oQ, ws=ws))
+                    others[name][f"dequant_{out_t}_ms"] = q_ms
+                    others[name][f"dequant_{out_t}_dense_equiv_tflops"] = oc.dense_equiv_flop / (q_ms * 1e-3) / 1e12
+                    del oQ
             del oA, oB, ovals, ometa, opruned, oD
         del flush
 

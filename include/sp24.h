@@ -160,6 +160,23 @@ sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A,
                       const void* meta, const void* B, const void* beta, const void* C,
                       void* D, void* workspace, size_t workspace_bytes, void* stream);
 
+/* INT8 sparse GEMM with a dequantising epilogue, for the deployment the paper describes in
+ * Section 4.4 and Section 5.1: INT8 weights and activations, per-row scaling factors for the
+ * weights of fully-connected layers and a per-tensor factor for the activations.
+ *   D[i,j] = act( row_scale[i] * acc[i,j] + bias[i] ),   acc = INT32 result of the 2:4 product,
+ * where row_scale[i] is the caller's product of the weight row's factor and the activation
+ * tensor's factor, bias may be NULL (0) and act is the identity or max(., 0) (relu != 0).
+ *   d->ab_type must be SP24_I8; d->cd_type: SP24_BF16, SP24_F16, SP24_F32, or SP24_I8.
+ *   SP24_I8 output: q = round-to-nearest-even(D / out_scale) clamped to [-127, 127].
+ *   row_scale, bias: device, M floats.  Everything is computed in FP32 in this order: acc to
+ *   float, one fused multiply-add with scale and bias, the activation, one multiply by
+ *   1/out_scale (rounded to float once on the host), the rounding.
+ * Other arguments, layouts and the workspace are those of sp24_gemm (alpha, beta, C unused). */
+sp24_status sp24_gemm_i8_dequant(const sp24_gemm_desc* d, const void* A, const void* meta,
+                                 const void* B, const float* row_scale, const float* bias,
+                                 int relu, float out_scale, void* D, void* workspace,
+                                 size_t workspace_bytes, void* stream);
+
 /* Copies the status record of the last sp24_gemm that used `workspace` back to the host
  * (synchronises `stream`) and returns SP24_OK, or SP24_ERR_TIMEOUT if a bounded wait inside
  * the kernel expired (the kernel then returned early and D is incomplete). */

@@ -64,6 +64,8 @@ def _load():
         lib.oracle_gemm_dense.restype = None
         lib.oracle_gemm_abs.argtypes = [i32, i64, vp, i64, vp, vp, i64, i32, i64, i64, i64, i64, vp]
         lib.oracle_gemm_abs.restype = None
+        lib.oracle_dequant.argtypes = [i64, i64, vp, vp, vp, i32, ctypes.c_float, vp, vp]
+        lib.oracle_dequant.restype = None
         lib.oracle_im2col_nhwc_3x3.argtypes = [i32, i64, i64, i64, i64, vp, vp, i64]
         lib.oracle_im2col_nhwc_3x3.restype = None
         _lib = lib
@@ -205,6 +207,20 @@ def gemm_abs(vals, meta, Bt, dtype, rows=None, cols=None) -> np.ndarray:
                             _ptr(np.ascontiguousarray(meta)), _ptr(Bt), K, 1, i0, i1, j0, j1,
                             _ptr(out))
     return out
+
+
+def dequant(acc: np.ndarray, row_scale: np.ndarray, bias=None, relu=False, out_scale=1.0):
+    """Dequantising epilogue on an exact int32 accumulator window (rows of `acc` pair with row_scale):
+    returns (float64 result, int8 code quantised with fp32 decisions)."""
+    assert acc.dtype == np.int32 and acc.ndim == 2 and acc.flags.c_contiguous
+    rs = np.ascontiguousarray(row_scale, dtype=np.float32)
+    b = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32)
+    assert rs.shape == (acc.shape[0],) and (b is None or b.shape == rs.shape)
+    f = np.empty(acc.shape, dtype=np.float64)
+    q = np.empty(acc.shape, dtype=np.int8)
+    _load().oracle_dequant(acc.shape[0], acc.shape[1], _ptr(acc), _ptr(rs), _ptr(b), 1 if relu else 0,
+                           ctypes.c_float(out_scale), _ptr(f), _ptr(q))
+    return f, q
 
 
 def im2col_nhwc_3x3(x: np.ndarray, dtype: str) -> np.ndarray:

@@ -373,4 +373,40 @@ void oracle_im2col_nhwc_3x3(int dtype, int64_t Nb, int64_t H, int64_t W, int64_t
             }
 }
 
+/* ------------------------------------------------------------------------------------- */
+/* Dequantising epilogue of the INT8 deployment (Section 4.4; Section 5.1: per-row scaling  */
+/* factors for fully-connected weights, a per-tensor factor for activations).  acc is the    */
+/* exact INT32 product; row_scale[i] already contains the activation factor.                */
+/*   out_f64:  y = row_scale[i] * acc + bias[i] in double, then the activation.             */
+/*   out_i8 :  the quantised code.  A rounding decision has to be taken in one precision on */
+/*             both sides, and the method fixes none, so it is the kernel's: float(acc)     */
+/*             (round to nearest), one fused multiply-add, the activation, one multiply by  */
+/*             1/out_scale (itself rounded to float), round-half-to-even, clamp to +-127.   */
+/* ------------------------------------------------------------------------------------- */
+void oracle_dequant(int64_t rows, int64_t cols, const int32_t* acc, const float* row_scale,
+                    const float* bias, int relu, float out_scale, double* out_f64, int8_t* out_i8) {
+  const float inv = 1.0f / out_scale;
+  for (int64_t i = 0; i < rows; ++i) {
+    for (int64_t j = 0; j < cols; ++j) {
+      int32_t a = acc[i * cols + j];
+      float b = bias ? bias[i] : 0.0f;
+      if (out_f64) {
+        double y = (double)row_scale[i] * (double)a + (double)b;
+        if (relu && y < 0.0) y = 0.0;
+        out_f64[i * cols + j] = y;
+      }
+      if (out_i8) {
+        float t = (float)a;
+        float y = fmaf(row_scale[i], t, b);
+        if (relu && !(y > 0.0f)) y = 0.0f;
+        volatile float z = y * inv; /* volatile: one rounding to float, no wider intermediate */
+        float q = rintf(z);
+        if (q > 127.0f) q = 127.0f;
+        if (q < -127.0f) q = -127.0f;
+        out_i8[i * cols + j] = (int8_t)q;
+      }
+    }
+  }
+}
+
 int oracle_elem_size(int dtype) { return elem_size(dtype); }

@@ -30,7 +30,7 @@ _FROM_TORCH = {torch.float16: "f16", torch.bfloat16: "bf16", torch.int8: "i8", t
 EXPORTS = [
     "sp24_status_string", "sp24_values_bytes", "sp24_meta_bytes", "sp24_prune", "sp24_compress",
     "sp24_decompress", "sp24_gemm_workspace_bytes", "sp24_gemm", "sp24_gemm_status",
-    "sp24_im2col_nhwc_3x3", "sp24_pipeline_host", "sp24_gemm_static_ws",
+    "sp24_im2col_nhwc_3x3", "sp24_pipeline_host", "sp24_gemm_static_ws", "sp24_gemm_i8_dequant",
 ]
 
 
@@ -69,6 +69,9 @@ def _load() -> ctypes.CDLL:
     lib.sp24_gemm.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sp24_gemm_static_ws.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sp24_gemm_static_ws.restype = ci
+    lib.sp24_gemm_i8_dequant.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, ci, ctypes.c_float, vp, vp,
+                                         sz, vp]
+    lib.sp24_gemm_i8_dequant.restype = ci
     lib.sp24_gemm_status.argtypes = [vp, vp]
     lib.sp24_im2col_nhwc_3x3.argtypes = [ci, i64, i64, i64, i64, vp, vp, i64, vp]
     lib.sp24_pipeline_host.argtypes = [ctypes.POINTER(GemmDesc)] + [vp] * 13 + [sz, vp]
@@ -230,4 +233,23 @@ def gemm_static_ws(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor,
     a, b = _scalar(ab, alpha), _scalar(ab, beta)
     _check(lib.sp24_gemm_static_ws(ctypes.byref(desc), ctypes.byref(a), _ptr(A), _ptr(meta), _ptr(Bt),
                                    ctypes.byref(b), _ptr(C), _ptr(out), _stream()), "sp24_gemm_static_ws")
+    return out
+
+
+def gemm_i8_dequant(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor, row_scale: torch.Tensor, *,
+                    bias: torch.Tensor | None = None, relu: bool = False, out_scale: float = 1.0, cd: str = "bf16",
+                    out: torch.Tensor | None = None, a_is_dense: bool = False, ws: torch.Tensor | None = None,
+                    b_row_major: bool = False, cd_col_major: bool = False) -> torch.Tensor:
+    """sp24_gemm_i8_dequant: int8 sparse GEMM, D = act(row_scale[i] * acc + bias[i]) as cd (bf16/f16/f32/i8)."""
+    M = A.shape[0]
+    K = A.shape[1] if a_is_dense else 2 * A.shape[1]
+    N = Bt.shape[1] if b_row_major else Bt.shape[0]
+    if out is None:
+        out = torch.empty((N, M) if cd_col_major else (M, N), dtype=TORCH_DTYPE[cd], device=A.device)
+    ws = ws if ws is not None else workspace(A.device)
+    desc = make_desc("i8", cd, M, N, K, A.stride(0), Bt.stride(0), M if cd_col_major else N, out.stride(0),
+                     a_is_dense, b_row_major, cd_col_major)
+    _check(lib.sp24_gemm_i8_dequant(ctypes.byref(desc), _ptr(A), _ptr(meta), _ptr(Bt), _ptr(row_scale), _ptr(bias),
+                                    1 if relu else 0, ctypes.c_float(out_scale), _ptr(out), _ptr(ws), ws.numel(),
+                                    _stream()), "sp24_gemm_i8_dequant")
     return out

@@ -54,6 +54,12 @@ struct GemmParams {
   int32_t has_c;
   int32_t band;       // m-tiles per band of the tile sweep
   int32_t cd_col_major;  // C and D stored M-contiguous (the [tokens, out_features] layout)
+  // int8 dequantising epilogue (sp24_gemm_i8_dequant): out = act(row_scale[i] * acc + bias[i]),
+  // requantised with out_inv_scale when the output type is int8
+  int32_t dequant, relu;
+  const float* row_scale;
+  const float* bias;
+  float out_inv_scale;
 };
 
 template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK, bool B_MN>
@@ -154,6 +160,89 @@ __device__ __forceinline__ uint32_t make_idesc(bool sparse, bool b_mn_major, int
 __device__ __forceinline__ uint4* staged_unit(uint8_t* buf, int cs, int row, int v) {
   return cs == 2 ? reinterpret_cast<uint4*>(buf + row * 64 + ((v ^ ((row >> 1) & 3)) << 4))
                  : reinterpret_cast<uint4*>(buf + row * 128 + ((v ^ (row & 7)) << 4));
+}
+
+// Dequantising epilogue of the int8 path, all in fp32 and in exactly this order (the int8 output
+// is compared bit for bit): t = float(acc) (round to nearest), y = fma(scale, t, bias), optional
+// max(y, 0); int8 output: round-to-nearest-even of y * out_inv_scale, clamped to [-127, 127].
+__device__ __forceinline__ float dequant_value(uint32_t acc, float scale, float bias, int relu) {
+  float y = __fmaf_rn(scale, __int2float_rn((int)acc), bias);
+  return relu ? fmaxf(y, 0.f) : y;
+}
+__device__ __forceinline__ int requant_i8(float y, float inv) {
+  int q = __float2int_rn(__fmul_rn(y, inv));
+  return max(-127, min(127, q));
+}
+
+__device__ __forceinline__ void convert_row_dequant(const uint32_t (&r)[32], uint8_t* buf, int lane, const GemmParams& p,
+                                                    float scale, float bias) {
+  if (p.cd_type == SP24_F32) {
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+      float4 o = make_float4(dequant_value(r[4 * v], scale, bias, p.relu), dequant_value(r[4 * v + 1], scale, bias, p.relu),
+                             dequant_value(r[4 * v + 2], scale, bias, p.relu), dequant_value(r[4 * v + 3], scale, bias, p.relu));
+      *reinterpret_cast<float4*>(staged_unit(buf, 4, lane, v)) = o;
+    }
+  } else if (p.cd_type == SP24_I8) {
+    // rows of 32 bytes, no swizzle
+#pragma unroll
+    for (int v = 0; v < 2; ++v) {
+      uint32_t w[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          int q = requant_i8(dequant_value(r[16 * v + 4 * e + b], scale, bias, p.relu), p.out_inv_scale);
+          word |= ((uint32_t)q & 0xFFu) << (8 * b);
+        }
+        w[e] = word;
+      }
+      *reinterpret_cast<uint4*>(buf + lane * 32 + v * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  } else {
+    const bool bf = p.cd_type == SP24_BF16;
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      uint32_t ow[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float2 f = make_float2(dequant_value(r[8 * v + 2 * e], scale, bias, p.relu),
+                               dequant_value(r[8 * v + 2 * e + 1], scale, bias, p.relu));
+        if (bf) {
+          __nv_bfloat162 o = __float22bfloat162_rn(f);
+          ow[e] = *reinterpret_cast<uint32_t*>(&o);
+        } else {
+          __half2 o = __float22half2_rn(f);
+          ow[e] = *reinterpret_cast<uint32_t*>(&o);
+        }
+      }
+      *staged_unit(buf, 2, lane, v) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+    }
+  }
+}
+
+// Column-major output of the dequantising epilogue: box transposed in the staging buffer.
+__device__ __forceinline__ void convert_row_dequant_transposed(const uint32_t (&r)[32], uint8_t* buf, int lane,
+                                                               const GemmParams& p, float scale, float bias) {
+#pragma unroll
+  for (int n = 0; n < 32; ++n) {
+    const float y = dequant_value(r[n], scale, bias, p.relu);
+    if (p.cd_type == SP24_F32) {
+      *reinterpret_cast<float*>(buf + n * 128 + ((((lane >> 2) ^ (n & 7))) << 4) + (lane & 3) * 4) = y;
+    } else if (p.cd_type == SP24_I8) {
+      *reinterpret_cast<int8_t*>(buf + n * 32 + lane) = (int8_t)requant_i8(y, p.out_inv_scale);
+    } else {
+      uint16_t* u = reinterpret_cast<uint16_t*>(buf + n * 64 + ((((lane >> 3) ^ ((n >> 1) & 3))) << 4) + (lane & 7) * 2);
+      if (p.cd_type == SP24_BF16) {
+        __nv_bfloat16 o = __float2bfloat16_rn(y);
+        *u = *reinterpret_cast<uint16_t*>(&o);
+      } else {
+        __half o = __float2half_rn(y);
+        *u = *reinterpret_cast<uint16_t*>(&o);
+      }
+    }
+  }
 }
 
 // This thread's row of the box: out = alpha * acc + beta * c, written over c in the staging buffer.
@@ -441,7 +530,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
     const int cs = elem_bytes((sp24_dtype)p.cd_type);
     const int buf_bytes = 1024 * cs;
-    const int nbuf = C::kEpiBytes / 4 / buf_bytes;  // staging buffers of this warp: 1, 2 or 4
+    const int nbuf = min(4, C::kEpiBytes / 4 / buf_bytes);  // staging buffers of this warp: 1, 2 or 4
     const int ahead = nbuf >= 4 ? 2 : 1;            // boxes the C loads run ahead
     // stores that may still be reading their buffer when the next buffer is claimed: with C the
     // buffer of box seq + ahead is claimed at the end of box seq, without C that of box seq + 1
@@ -515,8 +604,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int b = seq % nbuf;
         uint8_t* buf = my_bufs + b * buf_bytes;
         if (p.has_c && !bounded_wait(&sh->c_full[q][b], (seq / nbuf) & 1u, sh, p.status, 5u)) { ok = false; break; }
-        if (p.cd_col_major) convert_row_transposed<KIND>(r, buf, lane, p);
-        else convert_row<KIND>(r, buf, lane, p);
+        if (KIND == 1 && p.dequant) {
+          // this thread's output row: its scale and bias
+          const int row = min(row0 + lane, (int)p.M - 1);
+          const float scale = __ldg(p.row_scale + row), bias = p.bias ? __ldg(p.bias + row) : 0.f;
+          if (p.cd_col_major) convert_row_dequant_transposed(r, buf, lane, p, scale, bias);
+          else convert_row_dequant(r, buf, lane, p, scale, bias);
+        } else if (p.cd_col_major) {
+          convert_row_transposed<KIND>(r, buf, lane, p);
+        } else {
+          convert_row<KIND>(r, buf, lane, p);
+        }
         ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
@@ -691,11 +789,15 @@ extern "C" size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d) {
 
 static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A, const void* meta,
                                  const void* B, const void* beta, const void* C, void* D, void* ws, size_t ws_bytes,
-                                 bool& has_c, float& falpha, float& fbeta) {
-  SP24_RETURN_IF(d == nullptr || alpha == nullptr || beta == nullptr, SP24_ERR_NULL);
+                                 bool& has_c, float& falpha, float& fbeta, bool dequant = false) {
+  SP24_RETURN_IF(d == nullptr || (!dequant && (alpha == nullptr || beta == nullptr)), SP24_ERR_NULL);
   const bool fp = d->ab_type == SP24_F16 || d->ab_type == SP24_BF16;
   SP24_RETURN_IF(!fp && d->ab_type != SP24_I8, SP24_ERR_DTYPE);
-  if (fp) SP24_RETURN_IF(d->cd_type != d->ab_type && d->cd_type != SP24_F32, SP24_ERR_DTYPE);
+  if (dequant)
+    SP24_RETURN_IF(fp || (d->cd_type != SP24_BF16 && d->cd_type != SP24_F16 && d->cd_type != SP24_F32 &&
+                          d->cd_type != SP24_I8),
+                   SP24_ERR_DTYPE);
+  else if (fp) SP24_RETURN_IF(d->cd_type != d->ab_type && d->cd_type != SP24_F32, SP24_ERR_DTYPE);
   else SP24_RETURN_IF(d->cd_type != SP24_I32, SP24_ERR_DTYPE);
   const int64_t mult = fp ? 16 : 32;
   SP24_RETURN_IF(d->M < 0 || d->N < 0 || d->K <= 0, SP24_ERR_SHAPE);
@@ -703,7 +805,10 @@ static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, con
   SP24_RETURN_IF(d->M > (int64_t(1) << 30) || d->N > (int64_t(1) << 30) || d->K > (int64_t(1) << 30), SP24_ERR_SHAPE);
   SP24_RETURN_IF(d->order_b != SP24_COL_MAJOR && d->order_b != SP24_ROW_MAJOR, SP24_ERR_UNSUPPORTED);
   SP24_RETURN_IF(d->order_d != SP24_ROW_MAJOR && d->order_d != SP24_COL_MAJOR, SP24_ERR_UNSUPPORTED);
-  if (fp) {
+  if (dequant) {
+    falpha = 1.f;
+    fbeta = 0.f;
+  } else if (fp) {
     falpha = *static_cast<const float*>(alpha);
     fbeta = *static_cast<const float*>(beta);
   } else {
@@ -733,17 +838,32 @@ static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, con
   return SP24_OK;
 }
 
-extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A, const void* meta,
-                                 const void* B, const void* beta, const void* C, void* D, void* workspace,
-                                 size_t workspace_bytes, void* stream) {
+struct DequantArgs {
+  const float* row_scale;
+  const float* bias;
+  int relu;
+  float out_inv_scale;
+};
+
+static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A, const void* meta, const void* B,
+                            const void* beta, const void* C, void* D, void* workspace, size_t workspace_bytes,
+                            void* stream, const DequantArgs* dq) {
   bool has_c = false;
   float falpha = 1.f, fbeta = 0.f;
-  sp24_status st = validate_gemm(d, alpha, A, meta, B, beta, C, D, workspace, workspace_bytes, has_c, falpha, fbeta);
+  sp24_status st = validate_gemm(d, alpha, A, meta, B, beta, C, D, workspace, workspace_bytes, has_c, falpha, fbeta,
+                                 dq != nullptr);
   if (st != SP24_OK) return st;
   if (d->M == 0 || d->N == 0) return SP24_OK;
   if ((st = check_arch()) != SP24_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   GemmParams p = {};
+  if (dq) {
+    p.dequant = 1;
+    p.relu = dq->relu;
+    p.row_scale = dq->row_scale;
+    p.bias = dq->bias;
+    p.out_inv_scale = dq->out_inv_scale;
+  }
   p.M = d->M; p.N = d->N; p.K = d->K;
   p.ldc = d->ldc; p.ldd = d->ldd;
   p.C = has_c ? C : nullptr;
@@ -793,6 +913,22 @@ extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, con
 #undef SP24_DISPATCH_MN
 #undef SP24_LAUNCH
   return SP24_ERR_UNSUPPORTED;
+}
+
+extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A, const void* meta,
+                                 const void* B, const void* beta, const void* C, void* D, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+  return run_gemm(d, alpha, A, meta, B, beta, C, D, workspace, workspace_bytes, stream, nullptr);
+}
+
+extern "C" sp24_status sp24_gemm_i8_dequant(const sp24_gemm_desc* d, const void* A, const void* meta, const void* B,
+                                            const float* row_scale, const float* bias, int relu, float out_scale,
+                                            void* D, void* workspace, size_t workspace_bytes, void* stream) {
+  SP24_RETURN_IF(d == nullptr, SP24_ERR_NULL);
+  SP24_RETURN_IF(d->M > 0 && d->N > 0 && row_scale == nullptr, SP24_ERR_NULL);
+  SP24_RETURN_IF(d->cd_type == SP24_I8 && !(out_scale > 0.f), SP24_ERR_UNSUPPORTED);
+  DequantArgs dq = {row_scale, bias, relu ? 1 : 0, d->cd_type == SP24_I8 ? 1.0f / out_scale : 1.0f};
+  return run_gemm(d, nullptr, A, meta, B, nullptr, nullptr, D, workspace, workspace_bytes, stream, &dq);
 }
 
 extern "C" sp24_status sp24_gemm_status(const void* workspace, void* stream) {

@@ -188,6 +188,40 @@ def test_c_and_d_stored_m_contiguous(sp, case):
         check_fp(got, ref, scale, beta_c)
 
 
+@pytest.mark.parametrize("cd", ["bf16", "f16", "f32", "i8"])
+@pytest.mark.parametrize("layout", ["row", "col"])
+def test_int8_dequant_epilogue(sp, cd, layout):
+    """sp24_gemm_i8_dequant: float outputs within tolerance of the fp64 oracle, int8 codes bit-exact."""
+    cfg = inputs.scaled(inputs.CONFIGS["int8_linear"], M=416, N=608, K=1024)
+    M, N, K = cfg.M, cfg.N, cfg.K
+    A, Bt = inputs.gen_A(cfg), inputs.gen_Bt(cfg)
+    vals_ref, meta_ref, _ = oracle.compress(A, "i8")
+    acc = oracle.gemm_sparse(vals_ref, meta_ref, Bt, "i8")
+    rng = np.random.default_rng(17)
+    rs = (rng.uniform(0.5, 2.0, size=M) / (127.0 * 127.0 * np.sqrt(K / 2) / 3)).astype(np.float32)
+    bias = rng.normal(scale=0.5, size=M).astype(np.float32)
+    out_scale = 2.5 / 127.0
+    vals, meta, _ = sp.compress(to_device(A, "i8"))
+    for relu in (False, True):
+        D = sp.gemm_i8_dequant(vals, meta, to_device(Bt, "i8"), torch.from_numpy(rs).cuda(),
+                               bias=torch.from_numpy(bias).cuda(), relu=relu, out_scale=out_scale, cd=cd,
+                               cd_col_major=(layout == "col"))
+        torch.cuda.synchronize()
+        got = D.t() if layout == "col" else D
+        f_ref, q_ref = oracle.dequant(acc, rs, bias, relu=relu, out_scale=out_scale)
+        if cd == "i8":
+            assert np.array_equal(got.cpu().numpy(), q_ref)
+        else:
+            err = np.abs(to_host_f64(got) - f_ref)
+            tol = {"bf16": 2.0 ** -8, "f16": 2.0 ** -11, "f32": 2.0 ** -22}[cd]
+            bound = tol * (np.abs(rs.astype(np.float64))[:, None] * np.abs(acc) + np.abs(bias)[:, None]) + 1e-30
+            assert (err <= bound).all(), float((err / bound).max())
+    # no bias, fp32 out, scale 1: the integer accumulator itself while it is exactly representable
+    D = sp.gemm_i8_dequant(vals, meta, to_device(Bt, "i8"), torch.ones(M, device="cuda"), cd="f32")
+    torch.cuda.synchronize()
+    assert np.array_equal(to_host_f64(D), acc.astype(np.float32).astype(np.float64))
+
+
 def test_leading_dimensions_larger_than_the_matrices(sp):
     """Every operand as a window of a wider allocation (lda, ldb, ldc, ldd > logical width)."""
     cfg = inputs.scaled(inputs.CONFIGS["gpt3_ffn_bf16"], M=272, N=464, K=528)

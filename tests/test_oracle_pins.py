@@ -333,3 +333,35 @@ def test_operand_order_is_a_padded_bijection(dtype):
     hw = np.bincount(nib, minlength=16)
     canon[4] += buf.size * 2 - meta.size * 2
     assert np.array_equal(canon, hw)
+
+
+# ---------------------------------------------------------------------------------------
+# dequantising epilogue (Section 4.4, Section 5.1)
+# ---------------------------------------------------------------------------------------
+def test_dequant_closed_forms_and_numpy_float32():
+    rng = np.random.default_rng(3)
+    acc = rng.integers(-40_000_000, 40_000_000, size=(6, 50), dtype=np.int64).astype(np.int32)
+    acc[0, :8] = [0, 1, -1, 3, -3, 127, -127, 2**24 + 1]
+    ones = np.ones(6, np.float32)
+    f, q = oracle.dequant(acc, ones)                       # scale 1, no bias: identity / saturation
+    assert np.array_equal(f, acc.astype(np.float64))
+    assert np.array_equal(q[0, :7], [0, 1, -1, 3, -3, 127, -127]) and q[0, 7] == 127
+    f, q = oracle.dequant(acc, ones, relu=True)
+    assert np.array_equal(f, np.maximum(acc, 0).astype(np.float64)) and (q >= 0).all()
+    # halves round to even: acc * 0.5 with out_scale 1
+    half = np.array([[1, 3, 5, -1, -3, 7]], dtype=np.int32)
+    _, q = oracle.dequant(half, np.array([0.5], np.float32))
+    assert q.tolist() == [[0, 2, 2, 0, -2, 4]]
+    # general case against numpy float32 arithmetic (an independent library evaluation)
+    rs = rng.uniform(1e-6, 3e-6, size=6).astype(np.float32)
+    bias = rng.normal(size=6).astype(np.float32)
+    out_scale = np.float32(0.37)
+    f, q = oracle.dequant(acc, rs, bias, relu=True, out_scale=float(out_scale))
+    want64 = np.maximum(rs.astype(np.float64)[:, None] * acc + bias.astype(np.float64)[:, None], 0)
+    assert np.array_equal(f, want64)
+    t = acc.astype(np.float32)
+    y64 = rs.astype(np.float64)[:, None] * t.astype(np.float64) + bias.astype(np.float64)[:, None]  # exact product+sum
+    y = np.maximum(y64.astype(np.float32), np.float32(0))                                          # = one fma rounding
+    z = (y * (np.float32(1) / out_scale)).astype(np.float32)
+    want_q = np.clip(np.rint(z), -127, 127).astype(np.int8)
+    assert np.array_equal(q, want_q)

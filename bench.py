@@ -339,6 +339,11 @@ def run_ours(args, cfg):
                             "dense_variant_ms": d_ms, "speedup_vs_dense_variant": d_ms / s_ms}
             if im2col_ms is not None:
                 others[name]["im2col_ms"] = im2col_ms
+                oD2 = torch.empty((oc.M, oc.N), dtype=tdt[oc.cd_type], device=dev)
+                c_ms = time_flushed(lambda: sp.conv3x3_nhwc(ovals, ometa, x, out=oD2, cd=oc.cd_type, ws=ws))
+                others[name]["implicit_conv_ms"] = c_ms
+                others[name]["implicit_conv_dense_equiv_tflops"] = oc.dense_equiv_flop / (c_ms * 1e-3) / 1e12
+                del oD2
             if oc.ab_type == "i8":
                 # the dequantising epilogue (per-row scales) with bf16 and int8 outputs
                 rs = torch.full((oc.M,), 1e-5, dtype=torch.float32, device=dev)

@@ -177,6 +177,22 @@ sp24_status sp24_gemm_i8_dequant(const sp24_gemm_desc* d, const void* A, const v
                                  int relu, float out_scale, void* D, void* workspace,
                                  size_t workspace_bytes, void* stream);
 
+/* 3x3, stride-1, pad-1 convolution of an NHWC activation with 2:4-sparse weights as an implicit
+ * GEMM (Section 4.2: a convolution's reduction dimension is C*R*S): the same kernel as sp24_gemm,
+ * but the B operand is read straight from the activation by im2col-mode TMA loads instead of
+ * from a materialised (Nb*H*W) x 9*Cin matrix.
+ *   d:  as for sp24_gemm with N = Nb*H*W output pixels (pixel (n,h,w) is column (n*H+h)*W+w) and
+ *       K = 9*Cin ordered (r, s, c), c fastest; d->M output channels; ldb ignored; order_b must
+ *       be SP24_COL_MAJOR.  With order_d = SP24_COL_MAJOR the output is NHWC ([pixels, M]).
+ *   x:  device, Nb x H x W x Cin, packed, 16-byte aligned, at least 128 KiB.
+ *   Cin must be a multiple of 128 (16-bit types) or 256 (int8).
+ *   A / meta / alpha / beta / C / D / workspace: as for sp24_gemm (a_is_dense selects the dense
+ *   variant with A = Kout x 9*Cin). */
+sp24_status sp24_conv3x3_nhwc(const sp24_gemm_desc* d, int64_t Nb, int64_t H, int64_t W, int64_t Cin,
+                              const void* alpha, const void* A, const void* meta, const void* x,
+                              const void* beta, const void* C, void* D, void* workspace,
+                              size_t workspace_bytes, void* stream);
+
 /* Copies the status record of the last sp24_gemm that used `workspace` back to the host
  * (synchronises `stream`) and returns SP24_OK, or SP24_ERR_TIMEOUT if a bounded wait inside
  * the kernel expired (the kernel then returned early and D is incomplete). */

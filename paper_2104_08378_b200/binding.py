@@ -31,6 +31,7 @@ EXPORTS = [
     "sp24_status_string", "sp24_values_bytes", "sp24_meta_bytes", "sp24_prune", "sp24_compress",
     "sp24_decompress", "sp24_gemm_workspace_bytes", "sp24_gemm", "sp24_gemm_status",
     "sp24_im2col_nhwc_3x3", "sp24_pipeline_host", "sp24_gemm_static_ws", "sp24_gemm_i8_dequant",
+    "sp24_conv3x3_nhwc",
 ]
 
 
@@ -72,6 +73,8 @@ def _load() -> ctypes.CDLL:
     lib.sp24_gemm_i8_dequant.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, ci, ctypes.c_float, vp, vp,
                                          sz, vp]
     lib.sp24_gemm_i8_dequant.restype = ci
+    lib.sp24_conv3x3_nhwc.argtypes = [ctypes.POINTER(GemmDesc), i64, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sp24_conv3x3_nhwc.restype = ci
     lib.sp24_gemm_status.argtypes = [vp, vp]
     lib.sp24_im2col_nhwc_3x3.argtypes = [ci, i64, i64, i64, i64, vp, vp, i64, vp]
     lib.sp24_pipeline_host.argtypes = [ctypes.POINTER(GemmDesc)] + [vp] * 13 + [sz, vp]
@@ -252,4 +255,26 @@ def gemm_i8_dequant(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor
     _check(lib.sp24_gemm_i8_dequant(ctypes.byref(desc), _ptr(A), _ptr(meta), _ptr(Bt), _ptr(row_scale), _ptr(bias),
                                     1 if relu else 0, ctypes.c_float(out_scale), _ptr(out), _ptr(ws), ws.numel(),
                                     _stream()), "sp24_gemm_i8_dequant")
+    return out
+
+
+def conv3x3_nhwc(A: torch.Tensor, meta: torch.Tensor | None, x: torch.Tensor, *, alpha=1.0, beta=0.0,
+                 C: torch.Tensor | None = None, out: torch.Tensor | None = None, cd: str | None = None,
+                 ab: str | None = None, a_is_dense: bool = False, ws: torch.Tensor | None = None,
+                 nhwc_out: bool = False) -> torch.Tensor:
+    """sp24_conv3x3_nhwc: x [Nb, H, W, Cin] -> D [Kout, Nb*H*W] (or NHWC [Nb*H*W, Kout] with nhwc_out)."""
+    ab = _dtype_of(A, ab)
+    Nb, H, W, Cin = x.shape
+    M = A.shape[0]
+    K, N = 9 * Cin, Nb * H * W
+    cd = cd or ("i32" if ab == "i8" else ab)
+    if out is None:
+        out = torch.empty((N, M) if nhwc_out else (M, N), dtype=TORCH_DTYPE[cd], device=A.device)
+    ws = ws if ws is not None else workspace(A.device)
+    desc = make_desc(ab, cd, M, N, K, A.stride(0), K, C.stride(0) if C is not None else (M if nhwc_out else N),
+                     out.stride(0), a_is_dense, False, nhwc_out)
+    a, b = _scalar(ab, alpha), _scalar(ab, beta)
+    _check(lib.sp24_conv3x3_nhwc(ctypes.byref(desc), Nb, H, W, Cin, ctypes.byref(a), _ptr(A), _ptr(meta), _ptr(x),
+                                 ctypes.byref(b), _ptr(C), _ptr(out), _ptr(ws), ws.numel(), _stream()),
+           "sp24_conv3x3_nhwc")
     return out

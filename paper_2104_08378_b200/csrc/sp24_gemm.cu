@@ -54,6 +54,8 @@ struct GemmParams {
   int32_t has_c;
   int32_t band;       // m-tiles per band of the tile sweep
   int32_t cd_col_major;  // C and D stored M-contiguous (the [tokens, out_features] layout)
+  // implicit 3x3 convolution: B is the im2col view of an NHWC activation (never materialised)
+  int32_t conv, conv_h, conv_w, conv_c;
   // int8 dequantising epilogue (sp24_gemm_i8_dequant): out = act(row_scale[i] * acc + bias[i]),
   // requantised with out_inv_scale when the output type is int8
   int32_t dequant, relu;
@@ -402,6 +404,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int live = min(MBLK, (int)((p.M - (int64_t)mt * MBLK * CTAS * kBlockM + CTAS * kBlockM - 1) /
                                          (CTAS * kBlockM)));
         const uint32_t tx_bytes = (uint32_t)((live * (C::kABlockBytes + C::kEBlockBytes) + C::kBBytes) * CTAS);
+        // implicit convolution: (image, row, column) of this CTA's first output pixel
+        int conv_n = 0, conv_p = 0, conv_q = 0;
+        if (p.conv) {
+          conv_n = col0 / (p.conv_h * p.conv_w);
+          const int rem = col0 - conv_n * p.conv_h * p.conv_w;
+          conv_p = rem / p.conv_w;
+          conv_q = rem - conv_p * p.conv_w;
+        }
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!bounded_wait(&sh->empty[stage], phase ^ 1u, sh, p.status, 1u)) break;
           if (kb == hint_kb) sh->c_hint_tiles = tiles_started;
@@ -435,6 +445,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               int x = col0 + c * C::kBChunkElems, y = kb * C::kKPerStage;
               if (CTAS == 1) ptx::tma_load_2d(sb + c * C::kBChunkBytes, &map_b, full, x, y);
               else ptx::tma_load_2d_pair(sb + c * C::kBChunkBytes, &map_b, full, 0, x, y);
+            }
+          } else if (p.conv) {
+            // k = (r * 3 + s) * C + c: a stage holds channels of one filter tap; rows = output pixels
+            const int k0 = kb * C::kKPerStage;
+            const int tap = k0 / p.conv_c, c0 = k0 - tap * p.conv_c;
+            const int r = tap / 3, sx = tap - 3 * r;
+#pragma unroll
+            for (int i = 0; i < C::kBBoxes; ++i) {
+              uint8_t* dst = sb + i * C::kBRows * kAtomBytes;
+              if (CTAS == 1)
+                ptx::tma_load_im2col_4d(dst, &map_b, full, c0 + i * box_elems, conv_q - 1, conv_p - 1, conv_n,
+                                        (uint16_t)sx, (uint16_t)r);
+              else
+                ptx::tma_load_im2col_4d_pair(dst, &map_b, full, 0, c0 + i * box_elems, conv_q - 1, conv_p - 1, conv_n,
+                                             (uint16_t)sx, (uint16_t)r);
             }
           } else {
 #pragma unroll
@@ -678,6 +703,42 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+using EncodeIm2colFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*,
+                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                    CUtensorMapFloatOOBfill);
+
+EncodeIm2colFn encode_im2col_fn() {
+  static EncodeIm2colFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeIm2colFn>(ptr);
+  });
+  return fn;
+}
+
+// im2col tensor map over an NHWC activation for a 3x3, stride-1, pad-1 convolution: the bounding box
+// of the filter's anchor starts one pixel before the image and ends one pixel before its far edge, so
+// that anchor + tap (0..2) covers rows/columns -1 .. H, W with zeros outside.
+sp24_status make_im2col_map(CUtensorMap* map, const void* x, int es, uint64_t nb, uint64_t h, uint64_t w, uint64_t c,
+                            uint32_t channels_per_box, uint32_t pixels_per_box) {
+  EncodeIm2colFn fn = encode_im2col_fn();
+  if (!fn) return SP24_ERR_CUDA;
+  cuuint64_t dims[4] = {c, w, h, nb};
+  cuuint64_t strides[3] = {c * es, w * c * es, h * w * c * es};
+  int lower[2] = {-1, -1}, upper[2] = {-1, -1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUtensorMapDataType dt = es == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+  CUresult r = fn(map, dt, 4, const_cast<void*>(x), dims, strides, lower, upper, channels_per_box, pixels_per_box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SP24_OK : SP24_ERR_CUDA;
+}
+
 // 2-D tensor map over a row-major (rows x cols) array of `es`-byte elements with `ld_bytes`
 // between rows; box = box_cols x box_rows elements.
 sp24_status make_map(CUtensorMap* map, const void* base, int es, uint64_t rows, uint64_t cols, uint64_t ld_bytes,
@@ -723,8 +784,16 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
   const uint64_t a_cols = SPARSE ? d->K / 2 : d->K;
   sp24_status st = make_map(&map_a, A, es, d->M, a_cols, d->lda * es, atom_elems, kBlockM, 128);
   if (st != SP24_OK) return st;
-  if (B_MN) st = make_map(&map_b, B, es, d->K, d->N, d->ldb * es, C::kBChunkElems, C::kKPerStage, 128);
-  else st = make_map(&map_b, B, es, d->N, d->K, d->ldb * es, atom_elems, C::kBRows, 128);
+  if (p.conv) {
+    // B = im2col view of the NHWC activation: boxes of kBRows output pixels x one 128-byte run of channels
+    if (B_MN) return SP24_ERR_UNSUPPORTED;
+    const uint64_t nb = (uint64_t)d->N / ((uint64_t)p.conv_h * p.conv_w);
+    st = make_im2col_map(&map_b, B, es, nb, p.conv_h, p.conv_w, p.conv_c, atom_elems, C::kBRows);
+  } else if (B_MN) {
+    st = make_map(&map_b, B, es, d->K, d->N, d->ldb * es, C::kBChunkElems, C::kKPerStage, 128);
+  } else {
+    st = make_map(&map_b, B, es, d->N, d->K, d->ldb * es, atom_elems, C::kBRows, 128);
+  }
   if (st != SP24_OK) return st;
   if (SPARSE) {
     uint64_t meta_rows = (uint64_t)((d->M + 127) / 128) * p.meta_kb * 16;  // rows of 128 bytes
@@ -838,6 +907,10 @@ static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, con
   return SP24_OK;
 }
 
+struct ConvArgs {
+  int64_t nb, h, w, c;
+};
+
 struct DequantArgs {
   const float* row_scale;
   const float* bias;
@@ -847,7 +920,7 @@ struct DequantArgs {
 
 static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A, const void* meta, const void* B,
                             const void* beta, const void* C, void* D, void* workspace, size_t workspace_bytes,
-                            void* stream, const DequantArgs* dq) {
+                            void* stream, const DequantArgs* dq, const ConvArgs* cv = nullptr) {
   bool has_c = false;
   float falpha = 1.f, fbeta = 0.f;
   sp24_status st = validate_gemm(d, alpha, A, meta, B, beta, C, D, workspace, workspace_bytes, has_c, falpha, fbeta,
@@ -857,6 +930,12 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   if ((st = check_arch()) != SP24_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   GemmParams p = {};
+  if (cv) {
+    p.conv = 1;
+    p.conv_h = (int)cv->h;
+    p.conv_w = (int)cv->w;
+    p.conv_c = (int)cv->c;
+  }
   if (dq) {
     p.dequant = 1;
     p.relu = dq->relu;
@@ -929,6 +1008,27 @@ extern "C" sp24_status sp24_gemm_i8_dequant(const sp24_gemm_desc* d, const void*
   SP24_RETURN_IF(d->cd_type == SP24_I8 && !(out_scale > 0.f), SP24_ERR_UNSUPPORTED);
   DequantArgs dq = {row_scale, bias, relu ? 1 : 0, d->cd_type == SP24_I8 ? 1.0f / out_scale : 1.0f};
   return run_gemm(d, nullptr, A, meta, B, nullptr, nullptr, D, workspace, workspace_bytes, stream, &dq);
+}
+
+extern "C" sp24_status sp24_conv3x3_nhwc(const sp24_gemm_desc* d, int64_t Nb, int64_t H, int64_t W, int64_t Cin,
+                                         const void* alpha, const void* A, const void* meta, const void* x,
+                                         const void* beta, const void* C, void* D, void* workspace,
+                                         size_t workspace_bytes, void* stream) {
+  SP24_RETURN_IF(d == nullptr, SP24_ERR_NULL);
+  SP24_RETURN_IF(Nb <= 0 || H <= 0 || W <= 0 || Cin <= 0, SP24_ERR_SHAPE);
+  SP24_RETURN_IF(d->N != Nb * H * W || d->K != 9 * Cin, SP24_ERR_SHAPE);
+  SP24_RETURN_IF(!is_ab_type(d->ab_type), SP24_ERR_DTYPE);
+  // a shared-memory stage holds 128 (16-bit) or 256 (int8) consecutive k = channels of ONE filter tap
+  const int64_t per_stage = d->ab_type == SP24_I8 ? 256 : 128;
+  SP24_RETURN_IF(Cin % per_stage != 0, SP24_ERR_SHAPE);
+  SP24_RETURN_IF(H > 32767 || W > 32767 || Nb > (int64_t(1) << 30), SP24_ERR_SHAPE);
+  SP24_RETURN_IF(d->order_b != SP24_COL_MAJOR, SP24_ERR_UNSUPPORTED);
+  // smaller activations trip a tensor-map restriction of current drivers
+  SP24_RETURN_IF(Nb * H * W * Cin * elem_bytes(d->ab_type) < 131072, SP24_ERR_UNSUPPORTED);
+  sp24_gemm_desc dd = *d;
+  dd.ldb = d->K;  // not used by the im2col view, but keeps the generic checks meaningful
+  ConvArgs cv = {Nb, H, W, Cin};
+  return run_gemm(&dd, alpha, A, meta, x, beta, C, D, workspace, workspace_bytes, stream, nullptr, &cv);
 }
 
 extern "C" sp24_status sp24_gemm_status(const void* workspace, void* stream) {

@@ -109,3 +109,11 @@ def test_config5_resnet_conv_f16(sp):
     assert np.array_equal(to_host_bits(Btd), Bt)
     del Btd
     _run_config(sp, cfg, Bt, full_gemm=False)
+    # the same layer as an implicit GEMM (activation read through im2col-mode TMA, B never built)
+    A = inputs.gen_A(cfg)
+    vals_ref, meta_ref, _ = oracle.compress(A, cfg.ab_type)
+    vals, meta, _ = sp.compress(to_device(A, cfg.ab_type))
+    D = sp.conv3x3_nhwc(vals, meta, to_device(x, cfg.ab_type), cd=cfg.cd_type)
+    torch.cuda.synchronize()
+    assert sp.gemm_status(device=D.device) == 0
+    _check_tiles(cfg, D, vals_ref, meta_ref, Bt, None, _tiles(cfg, 64))

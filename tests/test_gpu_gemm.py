@@ -222,6 +222,43 @@ def test_int8_dequant_epilogue(sp, cd, layout):
     assert np.array_equal(to_host_f64(D), acc.astype(np.float32).astype(np.float64))
 
 
+@pytest.mark.parametrize("case", [("f16", 8, 14, 14, 128, 256), ("bf16", 5, 8, 20, 256, 144), ("i8", 8, 14, 14, 256, 288),
+                                  ("f16", 40, 14, 14, 128, 512)])
+@pytest.mark.parametrize("dense", [False, True])
+def test_implicit_conv3x3_matches_im2col_gemm(sp, case, dense):
+    """sp24_conv3x3_nhwc reads the activation through im2col-mode TMA: same result as the oracle's
+    explicit im2col followed by its sparse GEMM; NHWC output checked too."""
+    ab, Nb, H, W, Cin, Kout = case
+    dist = ("int8",) if ab == "i8" else ("relu_normal", 1.0)
+    x = inputs._matrix(dist, ab, 21, 1, H * W * Cin, 0, Nb).reshape(Nb, H, W, Cin)
+    wdist = ("int8",) if ab == "i8" else ("normal", float(np.sqrt(2.0 / (9 * Cin))))
+    A = inputs._matrix(wdist, ab, 21, 0, 9 * Cin, 0, Kout)
+    Bt = oracle.im2col_nhwc_3x3(np.ascontiguousarray(x), ab)
+    vals_ref, meta_ref, _ = oracle.compress(A, ab)
+    N = Nb * H * W
+    cols = (max(0, N - 400), N)
+    rows = (0, min(Kout, 160))
+    ref = oracle.gemm_sparse(vals_ref, meta_ref, Bt, ab, rows=rows, cols=cols)
+    ref0 = oracle.gemm_sparse(vals_ref, meta_ref, Bt, ab, rows=rows, cols=(0, 300))
+    Ad, xd = to_device(A, ab), to_device(x, ab)
+    cd = "i32" if ab == "i8" else "f32"
+    for nhwc in (False, True):
+        if dense:
+            D = sp.conv3x3_nhwc(sp.prune(Ad), None, xd, cd=cd, a_is_dense=True, nhwc_out=nhwc)
+        else:
+            vals, meta, _ = sp.compress(Ad)
+            D = sp.conv3x3_nhwc(vals, meta, xd, cd=cd, nhwc_out=nhwc)
+        torch.cuda.synchronize()
+        assert sp.gemm_status(device=D.device) == 0
+        Dm = D.t() if nhwc else D
+        for (c0, c1), want in ((cols, ref), ((0, 300), ref0)):
+            got = to_host_f64(Dm[rows[0]:rows[1], c0:c1])
+            if ab == "i8":
+                assert np.array_equal(got, want)
+            else:
+                check_fp(got, want, oracle.gemm_abs(vals_ref, meta_ref, Bt, ab, rows=rows, cols=(c0, c1)))
+
+
 def test_leading_dimensions_larger_than_the_matrices(sp):
     """Every operand as a window of a wider allocation (lda, ldb, ldc, ldd > logical width)."""
     cfg = inputs.scaled(inputs.CONFIGS["gpt3_ffn_bf16"], M=272, N=464, K=528)

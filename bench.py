@@ -355,7 +355,20 @@ def run_ours(args, cfg):
                     others[name][f"dequant_{out_t}_dense_equiv_tflops"] = oc.dense_equiv_flop / (q_ms * 1e-3) / 1e12
                     del oQ
             del oA, oB, ovals, ometa, opruned, oD
-        del flush
+        # TF32 mode with the 1:2 pattern (Section 3.2, Table 1) on a 4096 x 8192 x 4096 problem
+        tA = (torch.randn(4096, 4096, device=dev) * 0.02)
+        tB = torch.randn(8192, 4096, device=dev)
+        tvals, tmeta, _ = sp.compress(tA)
+        tprun = sp.prune(tA)
+        tD = torch.empty((4096, 8192), dtype=torch.float32, device=dev)
+        t_s = time_flushed(lambda: sp.gemm(tvals, tmeta, tB, out=tD, ws=ws))
+        t_d = time_flushed(lambda: sp.gemm(tprun, None, tB, out=tD, a_is_dense=True, ws=ws))
+        tflop = 2.0 * 4096 * 8192 * 4096
+        others["tf32_1of2_4096x8192x4096"] = {
+            "gemm_ms": t_s, "gemm_dense_equiv_tflops": tflop / (t_s * 1e-3) / 1e12,
+            "frac_of_measured_dense_bf16": tflop / (t_s * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "dense_variant_ms": t_d, "speedup_vs_dense_variant": t_d / t_s}
+        del flush, tA, tB, tvals, tmeta, tprun, tD
 
     # ---- end to end through the host-buffer entry point (rank-local) ----
     import ctypes

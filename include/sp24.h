@@ -53,6 +53,9 @@ typedef enum {
   SP24_ERR_ARCH = 10        /* current device is not sm_100                                */
 } sp24_status;
 
+/* SP24_F32 as an OPERAND type selects the TF32 mode (Section 3.2, Table 1): FP32 storage, TF32
+ * multiplication, FP32 accumulation, and the 1:2 pattern -- one kept value in every aligned
+ * PAIR along K instead of two in every group of four. */
 typedef enum { SP24_F16 = 0, SP24_BF16 = 1, SP24_I8 = 2, SP24_F32 = 3, SP24_I32 = 4 } sp24_dtype;
 
 /* Metadata layouts.
@@ -63,7 +66,11 @@ typedef enum { SP24_F16 = 0, SP24_BF16 = 1, SP24_I8 = 2, SP24_F32 = 3, SP24_I32 
  * TCGEN05: the same nibbles permuted into the order the sm_100a sparse tensor-core
  *   instruction reads them from tensor memory, in 2048-byte blocks of 128 rows x 128 columns
  *   of A, rows padded to a multiple of 128 and K to a multiple of 256; padding nibbles are 0x4.
- *   This is the layout sp24_gemm consumes. */
+ *   This is the layout sp24_gemm consumes.
+ * SP24_F32 (1:2 pattern): one nibble per PAIR, 0x4 if the first value of the pair is kept, 0xE if
+ *   the second (the pair read as four 16-bit halves of which halves 0,1 or 2,3 survive).
+ *   CANONICAL: K/4 bytes per row.  TCGEN05: the placement of the 16-bit types with a nibble
+ *   standing for a pair: 2048-byte blocks of 128 rows x 64 columns, K padded to 128. */
 typedef enum { SP24_META_CANONICAL = 0, SP24_META_TCGEN05 = 1 } sp24_meta_layout;
 
 /* Which index of a matrix is contiguous in memory. */
@@ -87,6 +94,9 @@ size_t sp24_meta_bytes(sp24_dtype t, int64_t M, int64_t K, sp24_meta_layout l);
  * magnitudes: the lower column index is kept.  Magnitude is |x| for I8 (so -128 ranks as
  * 128) and the bit pattern without its sign bit for F16/BF16 (denormals are not flushed).
  *   t: SP24_F16, SP24_BF16 or SP24_I8.      M >= 0, K >= 0, K % 4 == 0.
+ *      SP24_F32: the 1:2 pattern -- the larger magnitude of every aligned pair is kept, equal
+ *      magnitudes keep the first (K % 8 == 0, 16-byte aligned pointers and rows required;
+ *      the same holds for sp24_compress / sp24_decompress, whose vals are then M x K/2 FP32).
  *   x: device, M x K row-major, leading dimension ldx >= K (elements).
  *   y: device, same shape, leading dimension ldy >= K; may be the same buffer as x.
  * Fastest when x, y are 16-byte aligned and ldx*sizeof(t), ldy*sizeof(t), K*sizeof(t) are
@@ -116,7 +126,9 @@ sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals
                             void* stream);
 
 /* Problem description of D = alpha * op(A) * B + beta * C  (Section 3.2, Figure 2).
- *   ab_type: SP24_F16 or SP24_BF16 (FP32 accumulate) or SP24_I8 (INT32 accumulate) -- the
+ *   ab_type: SP24_F16 or SP24_BF16 (FP32 accumulate), SP24_I8 (INT32 accumulate) or SP24_F32
+ *            (TF32 mode, 1:2 pattern, FP32 accumulate; cd_type SP24_F32 and K-contiguous B
+ *            only; inputs are used with their low 13 mantissa bits ignored) -- the
  *            operand/accumulator pairs of Table 1.
  *   cd_type: type of C and D.  F16/BF16 operands: SP24_F16, SP24_BF16 (ab_type's own) or
  *            SP24_F32.  I8 operands: SP24_I32.

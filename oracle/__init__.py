@@ -64,6 +64,18 @@ def _load():
         lib.oracle_gemm_dense.restype = None
         lib.oracle_gemm_abs.argtypes = [i32, i64, vp, i64, vp, vp, i64, i32, i64, i64, i64, i64, vp]
         lib.oracle_gemm_abs.restype = None
+        lib.oracle_prune_1of2.argtypes = [i64, i64, vp, i64, vp, i64]
+        lib.oracle_prune_1of2.restype = None
+        lib.oracle_compress_1of2.argtypes = [i64, i64, vp, i64, vp, i64, vp]
+        lib.oracle_compress_1of2.restype = i64
+        lib.oracle_decompress_1of2.argtypes = [i64, i64, vp, i64, vp, vp, i64]
+        lib.oracle_decompress_1of2.restype = None
+        lib.oracle_gemm_sparse_1of2.argtypes = [i64, vp, i64, vp, vp, i64, dbl, dbl, vp, i64, i64, i64, i64, i64, vp, vp]
+        lib.oracle_gemm_sparse_1of2.restype = None
+        lib.oracle_meta_operand_bytes_1of2.argtypes = [i64, i64]
+        lib.oracle_meta_operand_bytes_1of2.restype = i64
+        lib.oracle_meta_permute_1of2.argtypes = [i64, i64, vp, vp, i32]
+        lib.oracle_meta_permute_1of2.restype = None
         lib.oracle_dequant.argtypes = [i64, i64, vp, vp, vp, i32, ctypes.c_float, vp, vp]
         lib.oracle_dequant.restype = None
         lib.oracle_im2col_nhwc_3x3.argtypes = [i32, i64, i64, i64, i64, vp, vp, i64]
@@ -206,6 +218,72 @@ def gemm_abs(vals, meta, Bt, dtype, rows=None, cols=None) -> np.ndarray:
     _load().oracle_gemm_abs(DTYPE_CODE[dtype], K, _ptr(vals), K2,
                             _ptr(np.ascontiguousarray(meta)), _ptr(Bt), K, 1, i0, i1, j0, j1,
                             _ptr(out))
+    return out
+
+
+# ---- the 1:2 pattern of the TF32 mode: fp32 matrices travel as numpy.uint32 bit patterns ----
+def _check32(a, name):
+    if a.dtype != np.uint32 or a.ndim != 2 or not a.flags.c_contiguous:
+        raise ValueError(f"{name}: need a C-contiguous 2-D uint32 array (fp32 bit patterns)")
+    return a
+
+
+def prune_1of2(x: np.ndarray) -> np.ndarray:
+    """Keep the larger-magnitude value of every aligned pair along a row (ties: the first)."""
+    _check32(x, "x")
+    M, K = x.shape
+    y = np.empty_like(x)
+    _load().oracle_prune_1of2(M, K, _ptr(x), K, _ptr(y), K)
+    return y
+
+
+def compress_1of2(x: np.ndarray):
+    """Returns (vals M x K/2 uint32, meta M x K/4 uint8 canonical nibbles 0x4 / 0xE, dropped)."""
+    _check32(x, "x")
+    M, K = x.shape
+    assert K % 4 == 0
+    vals = np.empty((M, K // 2), dtype=np.uint32)
+    meta = np.empty((M, K // 4), dtype=np.uint8)
+    dropped = _load().oracle_compress_1of2(M, K, _ptr(x), K, _ptr(vals), K // 2, _ptr(meta))
+    return vals, meta, int(dropped)
+
+
+def decompress_1of2(vals: np.ndarray, meta: np.ndarray) -> np.ndarray:
+    _check32(vals, "vals")
+    M, K2 = vals.shape
+    y = np.empty((M, 2 * K2), dtype=np.uint32)
+    _load().oracle_decompress_1of2(M, 2 * K2, _ptr(vals), K2, _ptr(np.ascontiguousarray(meta)), _ptr(y), 2 * K2)
+    return y
+
+
+def gemm_sparse_1of2(vals, meta, Bt, alpha=1.0, beta=0.0, C=None, rows=None, cols=None):
+    """(D, |A|.|B|) in float64 on an output window; Bt is N x K uint32 bit patterns, C float32 M x N."""
+    _check32(vals, "vals")
+    _check32(Bt, "Bt")
+    M, K2 = vals.shape
+    K, N = 2 * K2, Bt.shape[0]
+    assert Bt.shape[1] == K and meta.shape == (M, K // 4)
+    i0, i1, j0, j1 = _window(M, N, rows, cols)
+    out = np.zeros((i1 - i0, j1 - j0), dtype=np.float64)
+    mag = np.zeros_like(out)
+    if C is not None:
+        assert C.dtype == np.float32 and C.shape == (M, N) and C.flags.c_contiguous
+    _load().oracle_gemm_sparse_1of2(K, _ptr(vals), K2, _ptr(np.ascontiguousarray(meta)), _ptr(Bt), K, float(alpha),
+                                    float(beta), _ptr(C), N, i0, i1, j0, j1, _ptr(out), _ptr(mag))
+    return out, mag
+
+
+def meta_to_operand_order_1of2(meta: np.ndarray) -> np.ndarray:
+    M, K4 = meta.shape
+    K = 4 * K4
+    out = np.empty(int(_load().oracle_meta_operand_bytes_1of2(M, K)), dtype=np.uint8)
+    _load().oracle_meta_permute_1of2(M, K, _ptr(np.ascontiguousarray(meta)), _ptr(out), 0)
+    return out
+
+
+def meta_from_operand_order_1of2(buf: np.ndarray, M: int, K: int) -> np.ndarray:
+    out = np.empty((M, K // 4), dtype=np.uint8)
+    _load().oracle_meta_permute_1of2(M, K, _ptr(np.ascontiguousarray(buf)), _ptr(out), 1)
     return out
 
 

@@ -374,6 +374,114 @@ void oracle_im2col_nhwc_3x3(int dtype, int64_t Nb, int64_t H, int64_t W, int64_t
 }
 
 /* ------------------------------------------------------------------------------------- */
+/* The 1:2 pattern of the TF32 mode (Section 3.2: with FP32 input/output the pattern becomes */
+/* 1:2, i.e. one kept value in every aligned pair; Table 1, TF32 row).                        */
+/* FP32 storage as bit patterns (uint32).  Selection: larger magnitude (bit pattern without  */
+/* the sign), equal magnitudes keep the lower index.  Compressed form: vals M x K/2 and one  */
+/* nibble per pair, 0x4 if the first element is kept, 0xE if the second: the pair seen as    */
+/* four 16-bit halves of which halves (0,1) or (2,3) are kept, the 2:4 code of Section 3.1.  */
+/* Canonical layout: pair g of row i in bits 4g..4g+3 of the row (K/4 bytes per row).        */
+/* ------------------------------------------------------------------------------------- */
+static int keep_second_of_pair(const uint32_t* x, int64_t idx) {
+  uint32_t k0 = x[idx] & 0x7FFFFFFFu, k1 = x[idx + 1] & 0x7FFFFFFFu;
+  return k1 > k0; /* tie -> first */
+}
+
+void oracle_prune_1of2(int64_t M, int64_t K, const uint32_t* x, int64_t ldx, uint32_t* y, int64_t ldy) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < M; ++i)
+    for (int64_t g = 0; g < K / 2; ++g) {
+      int second = keep_second_of_pair(x, i * ldx + 2 * g);
+      y[i * ldy + 2 * g] = second ? 0u : x[i * ldx + 2 * g];
+      y[i * ldy + 2 * g + 1] = second ? x[i * ldx + 2 * g + 1] : 0u;
+    }
+}
+
+int64_t oracle_compress_1of2(int64_t M, int64_t K, const uint32_t* x, int64_t ldx, uint32_t* vals, int64_t ldv,
+                             uint8_t* meta) {
+  int64_t dropped = 0;
+  memset(meta, 0, (size_t)(M * (K / 4)));
+  for (int64_t i = 0; i < M; ++i)
+    for (int64_t g = 0; g < K / 2; ++g) {
+      int second = keep_second_of_pair(x, i * ldx + 2 * g);
+      vals[i * ldv + g] = x[i * ldx + 2 * g + second];
+      uint8_t nibble = second ? 0xE : 0x4;
+      meta[i * (K / 4) + g / 2] |= (uint8_t)(nibble << (4 * (g % 2)));
+      if ((x[i * ldx + 2 * g + (1 - second)] & 0x7FFFFFFFu) != 0) ++dropped;
+    }
+  return dropped;
+}
+
+static int pair_kept_index(const uint8_t* meta, int64_t K, int64_t i, int64_t g) {
+  int nibble = (meta[i * (K / 4) + g / 2] >> (4 * (g % 2))) & 0xF;
+  return (nibble & 3) >> 1; /* halves (0,1) -> element 0, halves (2,3) -> element 1 */
+}
+
+void oracle_decompress_1of2(int64_t M, int64_t K, const uint32_t* vals, int64_t ldv, const uint8_t* meta, uint32_t* y,
+                            int64_t ldy) {
+  for (int64_t i = 0; i < M; ++i) {
+    for (int64_t k = 0; k < K; ++k) y[i * ldy + k] = 0u;
+    for (int64_t g = 0; g < K / 2; ++g) y[i * ldy + 2 * g + pair_kept_index(meta, K, i, g)] = vals[i * ldv + g];
+  }
+}
+
+static double f32_bits_to_double(uint32_t w) {
+  float f;
+  memcpy(&f, &w, sizeof f);
+  return (double)f;
+}
+
+/* D[i,j] = alpha * sum_g vals[i,g] * B[2g + e(i,g), j] + beta * C[i,j], doubles throughout; B as   */
+/* N rows of K values (K contiguous); C fp32 (row-major, ldc); out_abs receives sum |a||b|.         */
+void oracle_gemm_sparse_1of2(int64_t K, const uint32_t* vals, int64_t ldv, const uint8_t* meta, const uint32_t* Bt,
+                             int64_t ldb, double alpha, double beta, const float* C, int64_t ldc, int64_t i0,
+                             int64_t i1, int64_t j0, int64_t j1, double* out, double* out_abs) {
+  int64_t width = j1 - j0;
+#pragma omp parallel for schedule(dynamic, 4)
+  for (int64_t i = i0; i < i1; ++i)
+    for (int64_t j = j0; j < j1; ++j) {
+      double acc = 0.0, mag = 0.0;
+      for (int64_t g = 0; g < K / 2; ++g) {
+        int64_t k = 2 * g + pair_kept_index(meta, K, i, g);
+        double a = f32_bits_to_double(vals[i * ldv + g]), b = f32_bits_to_double(Bt[j * ldb + k]);
+        acc += a * b;
+        mag += fabs(a) * fabs(b);
+      }
+      double r = alpha * acc;
+      if (beta != 0.0 && C) r += beta * (double)C[i * ldc + j];
+      out[(i - i0) * width + (j - j0)] = r;
+      if (out_abs) out_abs[(i - i0) * width + (j - j0)] = mag;
+    }
+}
+
+/* Operand order of the 1:2 metadata: the same nibble placement as the 16-bit types (a block  */
+/* is 128 rows x 32 nibbles), but a nibble stands for a pair, so a block covers 64 columns    */
+/* and K is padded to a multiple of 128.                                                      */
+int64_t oracle_meta_operand_bytes_1of2(int64_t M, int64_t K) {
+  return ((M + 127) / 128) * (2 * ((K + 127) / 128)) * 2048;
+}
+
+void oracle_meta_permute_1of2(int64_t M, int64_t K, const uint8_t* src, uint8_t* dst, int direction) {
+  int64_t MB = (M + 127) / 128, KB = 2 * ((K + 127) / 128);
+  if (direction == 0) memset(dst, 0x44, (size_t)(MB * KB * 2048));
+  else memset(dst, 0, (size_t)(M * (K / 4)));
+  for (int64_t i = 0; i < M; ++i)
+    for (int64_t g = 0; g < K / 2; ++g) {
+      int64_t mb = i / 128, kb = g / 32;
+      int r = (int)(i % 128), q = (int)(g % 32);
+      int64_t bit = ((mb * KB + kb) * 2048) * 8 + operand_bit_in_block(0, r, q);
+      int64_t cbyte = i * (K / 4) + g / 2, obyte = bit / 8;
+      int cshift = 4 * (int)(g % 2), oshift = (int)(bit % 8);
+      if (direction == 0) {
+        int nibble = (src[cbyte] >> cshift) & 0xF;
+        dst[obyte] = (uint8_t)((dst[obyte] & ~(0xF << oshift)) | (nibble << oshift));
+      } else {
+        dst[cbyte] |= (uint8_t)(((src[obyte] >> oshift) & 0xF) << cshift);
+      }
+    }
+}
+
+/* ------------------------------------------------------------------------------------- */
 /* Dequantising epilogue of the INT8 deployment (Section 4.4; Section 5.1: per-row scaling  */
 /* factors for fully-connected weights, a per-tensor factor for activations).  acc is the    */
 /* exact INT32 product; row_scale[i] already contains the activation factor.                */

@@ -5,7 +5,8 @@
  *
  * kinds: 0 = N(0, p0) by Box-Muller, 1 = U(p0, p1), 2 = integers uniform in [-127, 127],
  *        3 = max(N(0, p0), 0).
- * dtype: 0 = fp16 bits, 1 = bf16 bits (both round-to-nearest-even), 2 = int8.
+ * dtype: 0 = fp16 bits, 1 = bf16 bits (both round-to-nearest-even), 2 = int8,
+ *        3 = fp32 bits holding a TF32-representable value (10 mantissa bits, round-to-nearest-even).
  */
 #include <math.h>
 #include <stdint.h>
@@ -38,6 +39,14 @@ static uint16_t float_to_bf16_rne(float f) {
   return (uint16_t)(bits >> 16);
 }
 
+static uint32_t float_to_tf32_rne(float f) {
+  uint32_t bits;
+  memcpy(&bits, &f, 4);
+  if ((bits & 0x7F800000u) == 0x7F800000u) return bits & 0xFFFFE000u;
+  bits += 0xFFFu + ((bits >> 13) & 1u);
+  return bits & 0xFFFFE000u;
+}
+
 static uint16_t double_to_half_rne(double d) {
   /* _Float16 conversion from double rounds once, to nearest even. */
   _Float16 h = (_Float16)d;
@@ -63,7 +72,8 @@ void sp24_inputs_fill(int kind, double p0, double p1, int dtype, uint64_t seed,
       v = p0 * sqrt(-2.0 * log(unit_open(a))) * cos(6.283185307179586476925 * unit_open(b));
       if (kind == 3 && v < 0.0) v = 0.0;
     }
-    if (dtype == 2) ((int8_t*)out)[n] = (int8_t)v;
+    if (dtype == 3) ((uint32_t*)out)[n] = float_to_tf32_rne((float)v);
+    else if (dtype == 2) ((int8_t*)out)[n] = (int8_t)v;
     else if (dtype == 1) ((uint16_t*)out)[n] = float_to_bf16_rne((float)v);
     else ((uint16_t*)out)[n] = double_to_half_rne(v);
   }

@@ -38,11 +38,18 @@ extern "C" const char* sp24_status_string(sp24_status s) {
 }
 
 extern "C" size_t sp24_values_bytes(sp24_dtype t, int64_t M, int64_t K) {
+  if (t == SP24_F32) return (M < 0 || K < 0 || K % 2 != 0) ? 0 : (size_t)M * (size_t)(K / 2) * 4;
   if (!is_ab_type(t) || M < 0 || K < 0 || K % 4 != 0) return 0;
   return (size_t)M * (size_t)(K / 2) * (size_t)elem_bytes(t);
 }
 
 extern "C" size_t sp24_meta_bytes(sp24_dtype t, int64_t M, int64_t K, sp24_meta_layout l) {
+  if (t == SP24_F32) {  // 1:2 pattern: one nibble per pair
+    if (M < 0 || K < 0 || K % 4 != 0) return 0;
+    if (l == SP24_META_CANONICAL) return (size_t)M * (size_t)(K / 4);
+    if (l == SP24_META_TCGEN05) return (size_t)((M + 127) / 128) * (size_t)((K + 127) / 128) * 4096;
+    return 0;
+  }
   if (!is_ab_type(t) || M < 0 || K < 0 || K % 8 != 0) return 0;
   if (l == SP24_META_CANONICAL) return (size_t)M * (size_t)(K / 8);
   if (l == SP24_META_TCGEN05) return (size_t)((M + 127) / 128) * (size_t)((K + 255) / 256) * 4096;

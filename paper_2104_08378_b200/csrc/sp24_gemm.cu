@@ -73,14 +73,15 @@ struct Cfg {
   static constexpr int kBRows = BLOCK_N / CTAS;                    // B rows (N) this CTA loads
   static constexpr int kABlockBytes = kABoxes * kBlockM * kAtomBytes;  // one m-block
   static constexpr int kABytes = MBLK * kABlockBytes;
-  static constexpr int kKPerStage = (KIND == 0 ? 64 : 128) * kBBoxes;  // logical K per stage
+  static constexpr int kAtomElems = KIND == 0 ? 64 : (KIND == 1 ? 128 : 32);  // elements per 128-byte row
+  static constexpr int kKPerStage = kAtomElems * kBBoxes;  // logical K per stage
   // B with N contiguous (MN-major operand): 128-byte chunks along N, each kKPerStage k-rows of 128 bytes
-  static constexpr int kBChunkElems = KIND == 0 ? 64 : 128;
+  static constexpr int kBChunkElems = kAtomElems;
   static constexpr int kBChunks = (kBRows + kBChunkElems - 1) / kBChunkElems;
   static constexpr int kBChunkBytes = kKPerStage * kAtomBytes;
-  static constexpr int kBKStepBytes = (SPARSE ? 2 : 1) * (KIND == 0 ? 16 : 32) * kAtomBytes;  // k-rows of one MMA
+  static constexpr int kBKStepBytes = (SPARSE ? 2 : 1) * (kAtomElems / 4) * kAtomBytes;  // k-rows of one MMA
   static constexpr int kBBytes = B_MN ? kBChunks * kBChunkBytes : kBBoxes * kBRows * kAtomBytes;
-  static constexpr int kEBlocks = SPARSE ? (KIND == 0 ? 1 : 2) : 0;  // 2048-byte metadata blocks per m-block and stage
+  static constexpr int kEBlocks = SPARSE ? (KIND == 1 ? 2 : 1) : 0;  // 2048-byte metadata blocks per m-block and stage
   static constexpr int kEBlockBytes = kEBlocks * 2048;
   static constexpr int kEBytes = MBLK * kEBlockBytes;
   static constexpr int kEAlloc = (kEBytes + 1023) / 1024 * 1024;
@@ -144,8 +145,8 @@ template <int KIND>
 __device__ __forceinline__ uint32_t make_idesc(bool sparse, bool b_mn_major, int a_fmt, int m, int n) {
   uint32_t d = 0;
   d |= (sparse ? 1u : 0u) << 2;
-  d |= (KIND == 0 ? 1u : 2u) << 4;                 // accumulator: fp32 / int32
-  uint32_t fmt = KIND == 0 ? (uint32_t)a_fmt : 1u;  // f16 = 0, bf16 = 1; int8: 1 = signed
+  d |= (KIND == 1 ? 2u : 1u) << 4;                 // accumulator: int32 / fp32
+  uint32_t fmt = KIND == 0 ? (uint32_t)a_fmt : (KIND == 1 ? 1u : 2u);  // f16 = 0, bf16 = 1, tf32 = 2; int8: 1 = signed
   d |= fmt << 7;
   d |= fmt << 10;
   d |= (b_mn_major ? 1u : 0u) << 16;               // A is always K-major
@@ -391,7 +392,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (ptx::elect_one()) {
       int stage = 0;
       uint32_t phase = 0, tiles_started = 0;
-      const int box_elems = KIND == 0 ? 64 : 128;  // elements per 128-byte atom row
+      const int box_elems = C::kAtomElems;  // elements per 128-byte atom row
       const int hint_kb = max(0, p.k_blocks - 24);  // when the epilogue warps should pull C into the L2
       for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
         ++tiles_started;
@@ -522,7 +523,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 uint64_t da = ptx::smem_desc(saj + k * 32, true, 1024);
                 uint64_t db = B_MN ? ptx::smem_desc(sb + k * C::kBKStepBytes, true, 1024, C::kBChunkBytes)
                                    : ptx::smem_desc(sb + (k >> 1) * C::kBRows * kAtomBytes + (k & 1) * 64, true, 1024);
-                if (KIND == 0) {
+                if (KIND != 1) {
                   // one 32-bit metadata column per instruction: even-aligned address + selector
                   ptx::mma_sparse<KIND, CTAS>(d_tmem, da, db, e_tmem + (k & ~1), idesc | (uint32_t)(k & 1), accumulate);
                 } else {
@@ -773,12 +774,13 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
                    cudaStream_t stream) {
   using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS, MBLK, B_MN>;
   GemmParams p = base;
-  const int es = KIND == 0 ? 2 : 1;
+  const int es = KIND == 0 ? 2 : (KIND == 1 ? 1 : 4);
   const int tile_m = kBlockM * CTAS * MBLK;
   p.m_tiles = (int)((d->M + tile_m - 1) / tile_m);
   p.n_tiles = (int)((d->N + BLOCK_N - 1) / BLOCK_N);
   p.k_blocks = (int)((d->K + C::kKPerStage - 1) / C::kKPerStage);
-  p.meta_kb = (int)(2 * ((d->K + 255) / 256));
+  // metadata blocks per 128-row block: 128 columns each (64 for the 1:2 pattern), an even number of them
+  p.meta_kb = KIND == 2 ? (int)(2 * ((d->K + 127) / 128)) : (int)(2 * ((d->K + 255) / 256));
   CUtensorMap map_a, map_b, map_e;
   const uint32_t atom_elems = kAtomBytes / es;
   const uint64_t a_cols = SPARSE ? d->K / 2 : d->K;
@@ -787,6 +789,7 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
   if (p.conv) {
     // B = im2col view of the NHWC activation: boxes of kBRows output pixels x one 128-byte run of channels
     if (B_MN) return SP24_ERR_UNSUPPORTED;
+    if (KIND == 2) return SP24_ERR_UNSUPPORTED;
     const uint64_t nb = (uint64_t)d->N / ((uint64_t)p.conv_h * p.conv_w);
     st = make_im2col_map(&map_b, B, es, nb, p.conv_h, p.conv_w, p.conv_c, atom_elems, C::kBRows);
   } else if (B_MN) {
@@ -860,8 +863,10 @@ static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, con
                                  const void* B, const void* beta, const void* C, void* D, void* ws, size_t ws_bytes,
                                  bool& has_c, float& falpha, float& fbeta, bool dequant = false) {
   SP24_RETURN_IF(d == nullptr || (!dequant && (alpha == nullptr || beta == nullptr)), SP24_ERR_NULL);
-  const bool fp = d->ab_type == SP24_F16 || d->ab_type == SP24_BF16;
+  const bool tf32 = d->ab_type == SP24_F32;
+  const bool fp = d->ab_type == SP24_F16 || d->ab_type == SP24_BF16 || tf32;
   SP24_RETURN_IF(!fp && d->ab_type != SP24_I8, SP24_ERR_DTYPE);
+  SP24_RETURN_IF(tf32 && (d->cd_type != SP24_F32 || d->order_b != SP24_COL_MAJOR), SP24_ERR_UNSUPPORTED);
   if (dequant)
     SP24_RETURN_IF(fp || (d->cd_type != SP24_BF16 && d->cd_type != SP24_F16 && d->cd_type != SP24_F32 &&
                           d->cd_type != SP24_I8),
@@ -954,7 +959,7 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   p.has_c = has_c ? 1 : 0;
   p.cd_col_major = d->order_d == SP24_COL_MAJOR ? 1 : 0;
   const bool sparse = !d->a_is_dense;
-  const bool i8 = d->ab_type == SP24_I8;
+  const bool i8 = d->ab_type == SP24_I8, tf32 = d->ab_type == SP24_F32;
   // Tile choice.  Large problems (at least six waves of tiles): a pair of CTAs with two m-blocks
   // each, 512 x 224 tiles: least operand traffic per flop.  Medium: a pair with one m-block, 256 x 224,
   // epilogue overlapped.  Small: single CTAs, 128 x 128.  (224: two fp32 accumulators plus the
@@ -977,7 +982,9 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
 #define SP24_LAUNCH(K_, BN, CT, MB, MN)                                                               \
   (sparse ? launch<K_, true, BN, CT, MB, MN>(d, p, A, meta, B, s) : launch<K_, false, BN, CT, MB, MN>(d, p, A, meta, B, s))
 #define SP24_DISPATCH(CT, BN, MB)                                                                     \
-  if (ctas == CT && block_n == BN && mblk == MB && !b_mn) return i8 ? SP24_LAUNCH(1, BN, CT, MB, false) : SP24_LAUNCH(0, BN, CT, MB, false);
+  if (ctas == CT && block_n == BN && mblk == MB && !b_mn && !tf32) return i8 ? SP24_LAUNCH(1, BN, CT, MB, false) : SP24_LAUNCH(0, BN, CT, MB, false);
+#define SP24_DISPATCH_TF32(CT, BN, MB)                                                                \
+  if (ctas == CT && block_n == BN && mblk == MB && !b_mn && tf32) return SP24_LAUNCH(2, BN, CT, MB, false);
 #define SP24_DISPATCH_MN(CT, BN, MB)                                                                  \
   if (ctas == CT && block_n == BN && mblk == MB && b_mn) return i8 ? SP24_LAUNCH(1, BN, CT, MB, true) : SP24_LAUNCH(0, BN, CT, MB, true);
   SP24_DISPATCH(1, 128, 1)
@@ -985,11 +992,15 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   SP24_DISPATCH(2, 224, 2)
   SP24_DISPATCH(2, 192, 2)
   SP24_DISPATCH(2, 256, 1)
+  SP24_DISPATCH_TF32(1, 128, 1)
+  SP24_DISPATCH_TF32(2, 224, 1)
+  SP24_DISPATCH_TF32(2, 224, 2)
   SP24_DISPATCH_MN(1, 128, 1)
   SP24_DISPATCH_MN(2, 224, 1)
   SP24_DISPATCH_MN(2, 224, 2)
 #undef SP24_DISPATCH
 #undef SP24_DISPATCH_MN
+#undef SP24_DISPATCH_TF32
 #undef SP24_LAUNCH
   return SP24_ERR_UNSUPPORTED;
 }

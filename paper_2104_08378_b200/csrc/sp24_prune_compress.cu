@@ -438,6 +438,88 @@ __global__ void __launch_bounds__(kThreads) im2col_3x3_kernel(const uint8_t* __r
   st_stream(out + pixel * row_bytes_out + rem * 16, v);
 }
 
+// ---- the 1:2 pattern of the TF32 mode (Section 3.2): fp32 storage, one kept value per aligned pair ----
+// Metadata: one nibble per pair, 0x4 = first kept, 0xE = second kept (the pair seen as four 16-bit
+// halves of which (0,1) or (2,3) survive); canonical K/4 bytes per row, or the operand order of the
+// 16-bit types with a nibble standing for a pair (a 2048-byte block = 128 rows x 64 columns).
+__device__ __forceinline__ bool keep_second(uint32_t a, uint32_t b) { return (b & 0x7FFFFFFFu) > (a & 0x7FFFFFFFu); }
+
+__global__ void __launch_bounds__(kThreads) prune_f32_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x, uint8_t* y,
+                                                             int64_t row_bytes_y, int64_t vpr, int64_t rows) {
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= vpr) return;
+  for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows; row += (int64_t)gridDim.y * blockDim.y) {
+    uint4 v = ld_stream(x + row * row_bytes_x + c * 16);
+    const bool s0 = keep_second(v.x, v.y), s1 = keep_second(v.z, v.w);
+    st_stream(y + row * row_bytes_y + c * 16, make_uint4(s0 ? 0u : v.x, s0 ? v.y : 0u, s1 ? 0u : v.z, s1 ? v.w : 0u));
+  }
+}
+
+// Work unit: 8 columns (four pairs) = 32 bytes in, 16 bytes of values and 16 bits of metadata out.
+template <bool HW>
+__global__ void __launch_bounds__(kThreads) compress_f32_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
+                                                                uint8_t* __restrict__ vals, int64_t row_bytes_v,
+                                                                uint8_t* __restrict__ meta, int64_t M, int64_t K,
+                                                                int64_t rows_pad, int64_t chunks_pad,
+                                                                unsigned long long* dropped) {
+  const uint32_t chunk = blockIdx.x * blockDim.x + threadIdx.x, chunks = (uint32_t)(K >> 3), KB = (uint32_t)(chunks_pad >> 3);
+  const uint32_t moff = HW ? (chunk >> 3) * 2048u + 128u * (chunk & 1u) + 4u * ((chunk >> 1) & 3u) : 2u * chunk;
+  uint32_t lost = 0;
+  for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows_pad;
+       row += (int64_t)gridDim.y * blockDim.y) {
+    if (chunk >= (uint32_t)chunks_pad) continue;
+    uint32_t mbits = 0x4444u;
+    if (row < M && chunk < chunks) {
+      const uint8_t* src = x + row * row_bytes_x + chunk * 32u;
+      const uint4 a = ld_stream(src), b = ld_stream(src + 16);
+      const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+      uint32_t out[4];
+      mbits = 0;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const bool sec = keep_second(w[2 * g], w[2 * g + 1]);
+        out[g] = sec ? w[2 * g + 1] : w[2 * g];
+        mbits |= (sec ? 0xEu : 0x4u) << (4 * g);
+        lost += ((sec ? w[2 * g] : w[2 * g + 1]) & 0x7FFFFFFFu) != 0;
+      }
+      st_stream(vals + row * row_bytes_v + chunk * 16u, make_uint4(out[0], out[1], out[2], out[3]));
+    }
+    const uint32_t r = (uint32_t)row & 127u;
+    uint8_t* mr = HW ? meta + (row >> 7) * ((int64_t)KB * 2048) + (16u * (r & 7u) + 2u * ((r >> 3) & 1u) + 256u * (r >> 4))
+                     : meta + row * (K >> 2);
+    *reinterpret_cast<uint16_t*>(mr + moff) = (uint16_t)mbits;
+  }
+  if (dropped != nullptr && lost) atomicAdd(dropped, (unsigned long long)lost);
+}
+
+template <bool HW>
+__global__ void __launch_bounds__(kThreads) decompress_f32_kernel(const uint8_t* __restrict__ vals, int64_t row_bytes_v,
+                                                                  const uint8_t* __restrict__ meta, uint8_t* __restrict__ y,
+                                                                  int64_t row_bytes_y, int64_t M, int64_t K,
+                                                                  int64_t chunks_pad) {
+  const uint32_t chunk = blockIdx.x * blockDim.x + threadIdx.x, chunks = (uint32_t)(K >> 3), KB = (uint32_t)(chunks_pad >> 3);
+  if (chunk >= chunks) return;
+  const uint32_t moff = HW ? (chunk >> 3) * 2048u + 128u * (chunk & 1u) + 4u * ((chunk >> 1) & 3u) : 2u * chunk;
+  for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < M; row += (int64_t)gridDim.y * blockDim.y) {
+    const uint32_t r = (uint32_t)row & 127u;
+    const uint8_t* mr = HW ? meta + (row >> 7) * ((int64_t)KB * 2048) + (16u * (r & 7u) + 2u * ((r >> 3) & 1u) + 256u * (r >> 4))
+                           : meta + row * (K >> 2);
+    const uint32_t mbits = *reinterpret_cast<const uint16_t*>(mr + moff);
+    const uint4 v = ld_stream(vals + row * row_bytes_v + chunk * 16u);
+    const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+    uint32_t w[8];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      const bool sec = (((mbits >> (4 * g)) & 3u) >> 1) != 0;
+      w[2 * g] = sec ? 0u : in[g];
+      w[2 * g + 1] = sec ? in[g] : 0u;
+    }
+    uint8_t* dst = y + row * row_bytes_y + chunk * 32u;
+    st_stream(dst, make_uint4(w[0], w[1], w[2], w[3]));
+    st_stream(dst + 16, make_uint4(w[4], w[5], w[6], w[7]));
+  }
+}
+
 inline unsigned blocks_for(int64_t total, int per_block) { return (unsigned)((total + per_block - 1) / per_block); }
 
 // Block shape and grid of the vectorised kernels for `units` work units per row and `rows` rows:
@@ -472,8 +554,37 @@ static sp24_status validate_matrix_args(sp24_dtype t, int64_t M, int64_t K, int6
 
 using namespace sp24;
 
+// FP32 storage = the 1:2 pattern of the TF32 mode; vectorised paths only (16-byte aligned, K % 8 == 0).
+static sp24_status validate_f32(int64_t M, int64_t K, const void* a, int64_t lda, const void* b, int64_t ldb_bytes_ok) {
+  SP24_RETURN_IF(M < 0 || K < 0 || K % 8 != 0, SP24_ERR_SHAPE);
+  (void)a; (void)lda; (void)b; (void)ldb_bytes_ok;
+  return SP24_OK;
+}
+
+static dim3 f32_grid(int64_t units, int64_t rows, dim3& block) {
+  block = dim3(256, 1, 1);
+  if (units <= 128) block = dim3(units <= 32 ? 32 : (units <= 64 ? 64 : 128), 1, 1);
+  block.y = kThreads / block.x;
+  int64_t gy = (rows + block.y - 1) / block.y;
+  if (gy > 32768) gy = 32768;
+  return dim3((unsigned)((units + block.x - 1) / block.x), (unsigned)gy, 1);
+}
+
 extern "C" sp24_status sp24_prune(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx, void* y,
                                   int64_t ldy, void* stream) {
+  if (t == SP24_F32) {
+    sp24_status sf = validate_f32(M, K, x, ldx, y, ldy);
+    if (sf != SP24_OK) return sf;
+    if (M == 0 || K == 0) return SP24_OK;
+    SP24_RETURN_IF(x == nullptr || y == nullptr, SP24_ERR_NULL);
+    SP24_RETURN_IF(ldx < K || ldy < K || ldx % 4 || ldy % 4, SP24_ERR_STRIDE);
+    SP24_RETURN_IF(!aligned16(x) || !aligned16(y), SP24_ERR_ALIGN);
+    if ((sf = check_arch()) != SP24_OK) return sf;
+    dim3 block, grid = f32_grid(K / 4, M, block);
+    prune_f32_kernel<<<grid, block, 0, static_cast<cudaStream_t>(stream)>>>((const uint8_t*)x, ldx * 4, (uint8_t*)y, ldy * 4,
+                                                                             K / 4, M);
+    return cuda_status(cudaGetLastError());
+  }
   sp24_status st = validate_matrix_args(t, M, K, 4);
   if (st != SP24_OK) return st;
   if (M == 0 || K == 0) return SP24_OK;
@@ -511,6 +622,27 @@ extern "C" sp24_status sp24_prune(sp24_dtype t, int64_t M, int64_t K, const void
 extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx, void* vals,
                                      int64_t ldv, void* meta, sp24_meta_layout l, unsigned long long* dropped,
                                      void* stream) {
+  if (t == SP24_F32) {
+    sp24_status sf = validate_f32(M, K, x, ldx, vals, ldv);
+    if (sf != SP24_OK) return sf;
+    SP24_RETURN_IF(l != SP24_META_CANONICAL && l != SP24_META_TCGEN05, SP24_ERR_UNSUPPORTED);
+    if (M == 0 || K == 0) return SP24_OK;
+    SP24_RETURN_IF(x == nullptr || vals == nullptr || meta == nullptr, SP24_ERR_NULL);
+    SP24_RETURN_IF(ldx < K || ldv < K / 2 || ldx % 4 || ldv % 4, SP24_ERR_STRIDE);
+    SP24_RETURN_IF(!aligned16(x) || !aligned16(vals) || !aligned16(meta), SP24_ERR_ALIGN);
+    if ((sf = check_arch()) != SP24_OK) return sf;
+    const bool hw = l == SP24_META_TCGEN05;
+    const int64_t rows_pad = hw ? (M + 127) / 128 * 128 : M, k_pad = hw ? (K + 127) / 128 * 128 : K;
+    dim3 block, grid = f32_grid(k_pad / 8, rows_pad, block);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (hw)
+      compress_f32_kernel<true><<<grid, block, 0, s>>>((const uint8_t*)x, ldx * 4, (uint8_t*)vals, ldv * 4, (uint8_t*)meta,
+                                                       M, K, rows_pad, k_pad / 8, dropped);
+    else
+      compress_f32_kernel<false><<<grid, block, 0, s>>>((const uint8_t*)x, ldx * 4, (uint8_t*)vals, ldv * 4, (uint8_t*)meta,
+                                                        M, K, rows_pad, k_pad / 8, dropped);
+    return cuda_status(cudaGetLastError());
+  }
   sp24_status st = validate_matrix_args(t, M, K, 8);
   if (st != SP24_OK) return st;
   SP24_RETURN_IF(l != SP24_META_CANONICAL && l != SP24_META_TCGEN05, SP24_ERR_UNSUPPORTED);
@@ -585,6 +717,27 @@ extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const v
 
 extern "C" sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals, int64_t ldv,
                                        const void* meta, sp24_meta_layout l, void* y, int64_t ldy, void* stream) {
+  if (t == SP24_F32) {
+    sp24_status sf = validate_f32(M, K, vals, ldv, y, ldy);
+    if (sf != SP24_OK) return sf;
+    SP24_RETURN_IF(l != SP24_META_CANONICAL && l != SP24_META_TCGEN05, SP24_ERR_UNSUPPORTED);
+    if (M == 0 || K == 0) return SP24_OK;
+    SP24_RETURN_IF(y == nullptr || vals == nullptr || meta == nullptr, SP24_ERR_NULL);
+    SP24_RETURN_IF(ldy < K || ldv < K / 2 || ldy % 4 || ldv % 4, SP24_ERR_STRIDE);
+    SP24_RETURN_IF(!aligned16(y) || !aligned16(vals) || !aligned16(meta), SP24_ERR_ALIGN);
+    if ((sf = check_arch()) != SP24_OK) return sf;
+    const bool hw = l == SP24_META_TCGEN05;
+    const int64_t k_pad = hw ? (K + 127) / 128 * 128 : K;
+    dim3 block, grid = f32_grid(K / 8, M, block);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (hw)
+      decompress_f32_kernel<true><<<grid, block, 0, s>>>((const uint8_t*)vals, ldv * 4, (const uint8_t*)meta, (uint8_t*)y,
+                                                         ldy * 4, M, K, k_pad / 8);
+    else
+      decompress_f32_kernel<false><<<grid, block, 0, s>>>((const uint8_t*)vals, ldv * 4, (const uint8_t*)meta, (uint8_t*)y,
+                                                          ldy * 4, M, K, k_pad / 8);
+    return cuda_status(cudaGetLastError());
+  }
   sp24_status st = validate_matrix_args(t, M, K, 8);
   if (st != SP24_OK) return st;
   SP24_RETURN_IF(l != SP24_META_CANONICAL && l != SP24_META_TCGEN05, SP24_ERR_UNSUPPORTED);

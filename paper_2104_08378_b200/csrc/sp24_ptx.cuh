@@ -198,7 +198,8 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t smem_addr, bool swizzle12
 }
 
 // ---- MMA -------------------------------------------------------------------------------------------
-// KIND 0: kind::f16 (fp16 / bf16 operands, fp32 accumulate); KIND 1: kind::i8 (int32 accumulate).
+// KIND 0: kind::f16 (fp16 / bf16 operands, fp32 accumulate); KIND 1: kind::i8 (int32 accumulate);
+// KIND 2: kind::tf32 (fp32 storage, tf32 multiply, fp32 accumulate).
 template <int KIND, int CTAS>
 __device__ __forceinline__ void mma_dense(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate) {
@@ -213,6 +214,14 @@ __device__ __forceinline__ void mma_dense(uint32_t d_tmem, uint64_t a_desc, uint
   else if (KIND == 1 && CTAS == 1)
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                  "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc),
+                 "r"(idesc), "r"(accumulate) : "memory");
+  else if (KIND == 2 && CTAS == 1)
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc),
+                 "r"(idesc), "r"(accumulate) : "memory");
+  else if (KIND == 2 && CTAS == 2)
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc),
                  "r"(idesc), "r"(accumulate) : "memory");
   else
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
@@ -234,6 +243,14 @@ __device__ __forceinline__ void mma_sparse(uint32_t d_tmem, uint64_t a_desc, uin
   else if (KIND == 1 && CTAS == 1)
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
                  "tcgen05.mma.sp.cta_group::1.kind::i8 [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"(d_tmem), "l"(a_desc),
+                 "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
+  else if (KIND == 2 && CTAS == 1)
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                 "tcgen05.mma.sp.cta_group::1.kind::tf32 [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"(d_tmem), "l"(a_desc),
+                 "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
+  else if (KIND == 2 && CTAS == 2)
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                 "tcgen05.mma.sp.cta_group::2.kind::tf32 [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"(d_tmem), "l"(a_desc),
                  "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
   else
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"

@@ -8,7 +8,8 @@ range of a matrix can be regenerated on its own, which is how sampled output til
 largest configuration are checked without materialising everything twice.
 
 Storage convention: fp16 / bf16 matrices are numpy.uint16 BIT PATTERNS (round-to-nearest-even
-from float64 / float32), int8 matrices are numpy.int8.
+from float64 / float32), int8 matrices are numpy.int8, "tf32" matrices are numpy.uint32 bit
+patterns of fp32 values that are exactly representable in TF32 (10 mantissa bits).
 
 The configurations stand in for trained networks the paper evaluates (BERT-base FFN,
 GPT-3-scale FFN with hidden size 12288, a ResNet-50 3x3 convolution, an INT8 linear layer as
@@ -28,7 +29,7 @@ TENSOR_A, TENSOR_B, TENSOR_C, TENSOR_TILES = 0, 1, 2, 3
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "csrc", "inputs_gen.c")
 _LIB = os.path.join(_HERE, "libsp24_inputs.so")
-_DTYPE = {"f16": 0, "bf16": 1, "i8": 2}
+_DTYPE = {"f16": 0, "bf16": 1, "i8": 2, "tf32": 3}
 _lib = None
 
 
@@ -137,7 +138,7 @@ _KIND = {"normal": 0, "uniform": 1, "int8": 2, "relu_normal": 3}
 def _matrix(dist, dtype, seed, tensor_id, ncols, row0, row1) -> np.ndarray:
     """Rows row0..row1-1 of a (?, ncols) matrix whose element (r, c) has linear index r*ncols+c."""
     nrows = row1 - row0
-    out = np.empty((nrows, ncols), dtype=np.int8 if dtype == "i8" else np.uint16)
+    out = np.empty((nrows, ncols), dtype=np.int8 if dtype == "i8" else (np.uint32 if dtype == "tf32" else np.uint16))
     if nrows == 0 or ncols == 0:
         return out
     p0 = float(dist[1]) if len(dist) > 1 else 0.0

@@ -34,7 +34,10 @@ def test_size_helpers_and_status_strings():
     assert sp.meta_bytes("bf16", 49152, 12288, sp.META_CANONICAL) == 75497472
     assert sp.meta_bytes("bf16", 49152, 12288, sp.META_TCGEN05) == 75497472   # already tile-aligned
     assert sp.meta_bytes("i8", 200, 640, sp.META_TCGEN05) == 2 * 3 * 4096     # padded to 256 x 768
-    assert sp.values_bytes("f32", 4, 8) == 0
+    assert sp.values_bytes("f32", 4, 8) == 4 * 4 * 4                     # 1:2 pattern: K/2 fp32 values per row
+    assert sp.meta_bytes("f32", 100, 200, sp.META_CANONICAL) == 100 * 50  # one nibble per pair
+    assert sp.meta_bytes("f32", 100, 200, sp.META_TCGEN05) == 1 * 2 * 4096
+    assert sp.values_bytes("i32", 4, 8) == 0
     assert sp.status_string(0) == "ok" and "shape" in sp.status_string(3)
 
 
@@ -43,7 +46,7 @@ def test_argument_errors_are_reported_before_touching_a_device():
     lib = sp.lib
     one = ctypes.c_void_p(16)
     assert lib.sp24_prune(sp.F16, 4, 6, one, 6, one, 6, None) == 3            # K % 4
-    assert lib.sp24_prune(sp.F32, 4, 8, one, 8, one, 8, None) == 2            # dtype
+    assert lib.sp24_prune(sp.I32, 4, 8, one, 8, one, 8, None) == 2            # dtype
     assert lib.sp24_prune(sp.F16, 4, 8, None, 8, one, 8, None) == 1           # null
     assert lib.sp24_prune(sp.F16, 4, 8, one, 4, one, 8, None) == 4            # ld < K
     assert lib.sp24_prune(sp.F16, 0, 8, None, 8, None, 8, None) == 0          # empty: nothing to do

@@ -102,7 +102,7 @@ def test_empty_and_bad_arguments(sp):
     with pytest.raises(sp.Sp24Error):
         sp.compress(torch.zeros((4, 12), dtype=torch.int8, device="cuda"))   # K % 8 != 0
     with pytest.raises(sp.Sp24Error):
-        sp.prune(torch.zeros((4, 8), dtype=torch.float32, device="cuda"), dtype="f32")
+        sp.prune(torch.zeros((4, 8), dtype=torch.int32, device="cuda"), dtype="i32")
 
 
 @pytest.mark.parametrize("dtype", ["f16", "i8"])

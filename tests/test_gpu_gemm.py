@@ -259,6 +259,35 @@ def test_implicit_conv3x3_matches_im2col_gemm(sp, case, dense):
                 check_fp(got, want, oracle.gemm_abs(vals_ref, meta_ref, Bt, ab, rows=rows, cols=(c0, c1)))
 
 
+def test_pipeline_host_entry_point(sp):
+    """sp24_pipeline_host: host buffers in, compress + GEMM on the device, D back in a host buffer."""
+    import ctypes
+    cfg = inputs.scaled(inputs.CONFIGS["gpt3_ffn_bf16"], M=384, N=448, K=512)
+    M, N, K = cfg.M, cfg.N, cfg.K
+    A, Bt, Cm = inputs.gen_A(cfg), inputs.gen_Bt(cfg), inputs.gen_C(cfg)
+    hA, hB, hC = (torch.from_numpy(a.view(np.int16)).pin_memory() for a in (A, Bt, Cm))
+    hD = torch.empty((M, N), dtype=torch.int16).pin_memory()
+    dA = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dV = torch.empty((M, K // 2), dtype=torch.bfloat16, device="cuda")
+    dM = torch.empty(sp.meta_bytes("bf16", M, K), dtype=torch.uint8, device="cuda")
+    dB = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
+    dC = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    dD = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    desc = sp.make_desc("bf16", "bf16", M, N, K, K // 2, K, N, N)
+    al, be = ctypes.c_float(1.0), ctypes.c_float(1.0)
+    vp = lambda t: ctypes.c_void_p(t.data_ptr())  # noqa: E731
+    st = sp.lib.sp24_pipeline_host(ctypes.byref(desc), ctypes.byref(al), vp(hA), vp(hB), ctypes.byref(be), vp(hC), vp(hD),
+                                   vp(dA), vp(dV), vp(dM), vp(dB), vp(dC), vp(dD), vp(ws), 256,
+                                   torch.cuda.current_stream().cuda_stream)
+    assert st == 0
+    torch.cuda.synchronize()
+    vals_ref, meta_ref, _ = oracle.compress(A, "bf16")
+    ref = oracle.gemm_sparse(vals_ref, meta_ref, Bt, "bf16", 1.0, 1.0, Cm, "bf16")
+    got = oracle.bits_to_float64(hD.numpy().view(np.uint16), "bf16")
+    check_fp(got, ref, oracle.gemm_abs(vals_ref, meta_ref, Bt, "bf16"), np.abs(oracle.bits_to_float64(Cm, "bf16")))
+
+
 def test_leading_dimensions_larger_than_the_matrices(sp):
     """Every operand as a window of a wider allocation (lda, ldb, ldc, ldd > logical width)."""
     cfg = inputs.scaled(inputs.CONFIGS["gpt3_ffn_bf16"], M=272, N=464, K=528)

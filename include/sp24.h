@@ -234,6 +234,34 @@ sp24_status sp24_gemm_static_ws(const sp24_gemm_desc* d, const void* alpha, cons
 sp24_status sp24_im2col_nhwc_3x3(sp24_dtype t, int64_t Nb, int64_t H, int64_t W, int64_t C,
                                  const void* in, void* out, int64_t ldo, void* stream);
 
+/* Figure of merit of a channel permutation (Section 4.1: permuting the columns of the weight
+ * matrix before pruning so that large values are spread over the groups keeps more total
+ * magnitude).  Adds to *result (device double) the sum of |x[i, perm[k]]| over the positions
+ * that 2:4 pruning of the column-permuted matrix x'[:, k] = x[:, perm[k]] keeps.
+ *   perm: device, K int32 column indices (a permutation of 0..K-1), or NULL for the identity.
+ *   t: SP24_F16, SP24_BF16, SP24_I8;  K % 4 == 0;  ldx >= K.  Summation is in double; the
+ *   order of the partial sums is not fixed. */
+sp24_status sp24_kept_magnitude(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx,
+                                const int32_t* perm, double* result, void* stream);
+
+/* Re-imposes a fixed 2:4 pattern on updated weights, as sparse retraining does (Section 4.1,
+ * step 3: the pattern found in step 2 is kept while the weights train on):
+ * y[i, k] = w[i, k] where the metadata of sp24_compress names k as kept, +0 elsewhere.
+ *   meta / l: metadata of an M x K matrix in either layout.  K % 8 == 0; y may alias w. */
+sp24_status sp24_apply_mask(sp24_dtype t, int64_t M, int64_t K, const void* w, int64_t ldw,
+                            const void* meta, sp24_meta_layout l, void* y, int64_t ldy,
+                            void* stream);
+
+/* 2:4 along rows AND columns (Section 6: the pattern must also hold for the transposed weights
+ * if the backward pass is to be accelerated).  Every aligned 4 x 4 block keeps exactly two
+ * values per row and per column; of the 90 such patterns the one keeping the largest total
+ * magnitude is taken (exhaustive search).  Score of a pattern: ((s0 + s1) + s2) + s3 with
+ * s_i = |x[i, c]| + |x[i, c']| for the row's kept columns c < c', in FP32; patterns are numbered
+ * lexicographically by their rows' kept pairs in the order 01, 02, 03, 12, 13, 23, and the
+ * lowest-numbered pattern with the largest score wins.  M % 4 == 0, K % 4 == 0; y may alias x. */
+sp24_status sp24_prune_2d(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx,
+                          void* y, int64_t ldy, void* stream);
+
 /* End-to-end convenience for callers whose data lives in HOST memory (pinned for speed):
  * copies dense A (M x K, row-major, packed), B (N rows of K, packed) and, if beta != 0, C
  * (M x N packed) to the device buffers the caller provides, runs sp24_compress (TCGEN05

@@ -76,6 +76,12 @@ def _load():
         lib.oracle_meta_operand_bytes_1of2.restype = i64
         lib.oracle_meta_permute_1of2.argtypes = [i64, i64, vp, vp, i32]
         lib.oracle_meta_permute_1of2.restype = None
+        lib.oracle_kept_magnitude.argtypes = [i32, i64, i64, vp, i64, vp]
+        lib.oracle_kept_magnitude.restype = dbl
+        lib.oracle_apply_mask.argtypes = [i32, i64, i64, vp, i64, vp, vp, i64]
+        lib.oracle_apply_mask.restype = None
+        lib.oracle_prune_2d.argtypes = [i32, i64, i64, vp, i64, vp, i64]
+        lib.oracle_prune_2d.restype = None
         lib.oracle_dequant.argtypes = [i64, i64, vp, vp, vp, i32, ctypes.c_float, vp, vp]
         lib.oracle_dequant.restype = None
         lib.oracle_im2col_nhwc_3x3.argtypes = [i32, i64, i64, i64, i64, vp, vp, i64]
@@ -285,6 +291,33 @@ def meta_from_operand_order_1of2(buf: np.ndarray, M: int, K: int) -> np.ndarray:
     out = np.empty((M, K // 4), dtype=np.uint8)
     _load().oracle_meta_permute_1of2(M, K, _ptr(np.ascontiguousarray(buf)), _ptr(out), 1)
     return out
+
+
+def kept_magnitude(x: np.ndarray, dtype: str, perm=None) -> float:
+    """Total magnitude kept by 2:4 pruning of x with its columns permuted by `perm` (Section 4.1)."""
+    _check(x, dtype, "x")
+    M, K = x.shape
+    p = None if perm is None else np.ascontiguousarray(perm, dtype=np.int32)
+    return float(_load().oracle_kept_magnitude(DTYPE_CODE[dtype], M, K, _ptr(x), K, _ptr(p)))
+
+
+def apply_mask(w: np.ndarray, meta: np.ndarray, dtype: str) -> np.ndarray:
+    """Keep w where the canonical metadata names the position, +0 elsewhere (Section 4.1 step 3)."""
+    _check(w, dtype, "w")
+    M, K = w.shape
+    y = np.empty_like(w)
+    _load().oracle_apply_mask(DTYPE_CODE[dtype], M, K, _ptr(w), K, _ptr(np.ascontiguousarray(meta)), _ptr(y), K)
+    return y
+
+
+def prune_2d(x: np.ndarray, dtype: str) -> np.ndarray:
+    """2:4 along rows and columns of every aligned 4 x 4 block, exhaustive search (Section 6)."""
+    _check(x, dtype, "x")
+    M, K = x.shape
+    assert M % 4 == 0 and K % 4 == 0
+    y = np.empty_like(x)
+    _load().oracle_prune_2d(DTYPE_CODE[dtype], M, K, _ptr(x), K, _ptr(y), K)
+    return y
 
 
 def dequant(acc: np.ndarray, row_scale: np.ndarray, bias=None, relu=False, out_scale=1.0):

@@ -517,4 +517,79 @@ void oracle_dequant(int64_t rows, int64_t cols, const int32_t* acc, const float*
   }
 }
 
+/* ------------------------------------------------------------------------------------- */
+/* Tools around the pruning step.                                                          */
+/* ------------------------------------------------------------------------------------- */
+/* Section 4.1 (channel permutations): total magnitude kept by 2:4 pruning of the matrix    */
+/* whose column k is column perm[k] of x (perm NULL = identity), summed in double.          */
+double oracle_kept_magnitude(int dtype, int64_t M, int64_t K, const void* x, int64_t ldx, const int32_t* perm) {
+  double total = 0.0;
+  for (int64_t i = 0; i < M; ++i)
+    for (int64_t g = 0; g < K / 4; ++g) {
+      int key[4], p0, p1;
+      int64_t idx[4];
+      for (int p = 0; p < 4; ++p) {
+        idx[p] = i * ldx + (perm ? perm[4 * g + p] : 4 * g + p);
+        key[p] = magnitude_key(dtype, x, idx[p]);
+      }
+      select_two(key, &p0, &p1);
+      total += fabs(load_as_double(dtype, x, idx[p0])) + fabs(load_as_double(dtype, x, idx[p1]));
+    }
+  return total;
+}
+
+/* Section 4.1 step 3: the pattern stays fixed while the weights change: keep w where the    */
+/* canonical metadata names the position, +0 elsewhere.                                       */
+void oracle_apply_mask(int dtype, int64_t M, int64_t K, const void* w, int64_t ldw, const uint8_t* meta, void* y,
+                       int64_t ldy) {
+  for (int64_t i = 0; i < M; ++i)
+    for (int64_t g = 0; g < K / 4; ++g) {
+      int p0, p1;
+      nibble_positions(meta, K, i, g, &p0, &p1);
+      for (int p = 0; p < 4; ++p) {
+        if (p == p0 || p == p1) copy_elem(dtype, y, i * ldy + 4 * g + p, w, i * ldw + 4 * g + p);
+        else zero_elem(dtype, y, i * ldy + 4 * g + p);
+      }
+    }
+}
+
+/* Section 6: 2:4 along rows and columns of every aligned 4 x 4 block.  All assignments of one of  */
+/* the six pairs {01,02,03,12,13,23} to each of the four rows are visited in lexicographic order;  */
+/* those whose columns all hold exactly two kept entries are the 90 candidates.  Which one is      */
+/* "largest" is a floating-point decision and the method fixes no precision, so it is the kernel's: */
+/* score = ((s0 + s1) + s2) + s3, s_i = |x[i,c]| + |x[i,c']|, all in float; the first candidate    */
+/* with the strictly largest score wins.                                                           */
+void oracle_prune_2d(int dtype, int64_t M, int64_t K, const void* x, int64_t ldx, void* y, int64_t ldy) {
+  static const int pair[6][2] = {{0, 1}, {0, 2}, {0, 3}, {1, 2}, {1, 3}, {2, 3}};
+  for (int64_t bi = 0; bi < M / 4; ++bi)
+    for (int64_t bj = 0; bj < K / 4; ++bj) {
+      float mag[4][4];
+      for (int i = 0; i < 4; ++i)
+        for (int j = 0; j < 4; ++j) mag[i][j] = (float)fabs(load_as_double(dtype, x, (4 * bi + i) * ldx + 4 * bj + j));
+      float best = -1.0f;
+      int best_rows[4] = {0, 0, 0, 0};
+      int r[4];
+      for (r[0] = 0; r[0] < 6; ++r[0])
+        for (r[1] = 0; r[1] < 6; ++r[1])
+          for (r[2] = 0; r[2] < 6; ++r[2])
+            for (r[3] = 0; r[3] < 6; ++r[3]) {
+              int col[4] = {0, 0, 0, 0};
+              for (int i = 0; i < 4; ++i) { ++col[pair[r[i]][0]]; ++col[pair[r[i]][1]]; }
+              if (col[0] != 2 || col[1] != 2 || col[2] != 2 || col[3] != 2) continue;
+              volatile float sc = 0.0f;
+              for (int i = 0; i < 4; ++i) {
+                volatile float si = mag[i][pair[r[i]][0]] + mag[i][pair[r[i]][1]];
+                sc = (i == 0) ? si : sc + si;
+              }
+              if (sc > best) { best = sc; for (int i = 0; i < 4; ++i) best_rows[i] = r[i]; }
+            }
+      for (int i = 0; i < 4; ++i)
+        for (int j = 0; j < 4; ++j) {
+          int keep = j == pair[best_rows[i]][0] || j == pair[best_rows[i]][1];
+          if (keep) copy_elem(dtype, y, (4 * bi + i) * ldy + 4 * bj + j, x, (4 * bi + i) * ldx + 4 * bj + j);
+          else zero_elem(dtype, y, (4 * bi + i) * ldy + 4 * bj + j);
+        }
+    }
+}
+
 int oracle_elem_size(int dtype) { return elem_size(dtype); }

@@ -31,7 +31,7 @@ EXPORTS = [
     "sp24_status_string", "sp24_values_bytes", "sp24_meta_bytes", "sp24_prune", "sp24_compress",
     "sp24_decompress", "sp24_gemm_workspace_bytes", "sp24_gemm", "sp24_gemm_status",
     "sp24_im2col_nhwc_3x3", "sp24_pipeline_host", "sp24_gemm_static_ws", "sp24_gemm_i8_dequant",
-    "sp24_conv3x3_nhwc",
+    "sp24_conv3x3_nhwc", "sp24_kept_magnitude", "sp24_apply_mask", "sp24_prune_2d",
 ]
 
 
@@ -75,6 +75,11 @@ def _load() -> ctypes.CDLL:
     lib.sp24_gemm_i8_dequant.restype = ci
     lib.sp24_conv3x3_nhwc.argtypes = [ctypes.POINTER(GemmDesc), i64, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sp24_conv3x3_nhwc.restype = ci
+    lib.sp24_kept_magnitude.argtypes = [ci, i64, i64, vp, i64, vp, vp, vp]
+    lib.sp24_apply_mask.argtypes = [ci, i64, i64, vp, i64, vp, ci, vp, i64, vp]
+    lib.sp24_prune_2d.argtypes = [ci, i64, i64, vp, i64, vp, i64, vp]
+    for name in ("sp24_kept_magnitude", "sp24_apply_mask", "sp24_prune_2d"):
+        getattr(lib, name).restype = ci
     lib.sp24_gemm_status.argtypes = [vp, vp]
     lib.sp24_im2col_nhwc_3x3.argtypes = [ci, i64, i64, i64, i64, vp, vp, i64, vp]
     lib.sp24_pipeline_host.argtypes = [ctypes.POINTER(GemmDesc)] + [vp] * 13 + [sz, vp]
@@ -277,4 +282,37 @@ def conv3x3_nhwc(A: torch.Tensor, meta: torch.Tensor | None, x: torch.Tensor, *,
     _check(lib.sp24_conv3x3_nhwc(ctypes.byref(desc), Nb, H, W, Cin, ctypes.byref(a), _ptr(A), _ptr(meta), _ptr(x),
                                  ctypes.byref(b), _ptr(C), _ptr(out), _ptr(ws), ws.numel(), _stream()),
            "sp24_conv3x3_nhwc")
+    return out
+
+
+def kept_magnitude(x: torch.Tensor, perm: torch.Tensor | None = None, dtype: str | None = None) -> torch.Tensor:
+    """sp24_kept_magnitude: total magnitude 2:4 pruning keeps under a column permutation (device double[1])."""
+    dt = _dtype_of(x, dtype)
+    M, K = x.shape
+    res = torch.zeros(1, dtype=torch.float64, device=x.device)
+    _check(lib.sp24_kept_magnitude(DTYPE_CODE[dt], M, K, _ptr(x), x.stride(0) if M > 1 else K, _ptr(perm), _ptr(res),
+                                   _stream()), "sp24_kept_magnitude")
+    return res
+
+
+def apply_mask(w: torch.Tensor, meta: torch.Tensor, layout: int = META_TCGEN05, out: torch.Tensor | None = None,
+               dtype: str | None = None) -> torch.Tensor:
+    """sp24_apply_mask: zero every position of w the metadata does not name as kept."""
+    dt = _dtype_of(w, dtype)
+    M, K = w.shape
+    if out is None:
+        out = torch.empty_like(w)
+    _check(lib.sp24_apply_mask(DTYPE_CODE[dt], M, K, _ptr(w), w.stride(0) if M > 1 else K, _ptr(meta), layout, _ptr(out),
+                               out.stride(0) if M > 1 else K, _stream()), "sp24_apply_mask")
+    return out
+
+
+def prune_2d(x: torch.Tensor, out: torch.Tensor | None = None, dtype: str | None = None) -> torch.Tensor:
+    """sp24_prune_2d: 2:4 along rows and columns of every 4 x 4 block (exhaustive search)."""
+    dt = _dtype_of(x, dtype)
+    M, K = x.shape
+    if out is None:
+        out = torch.empty_like(x)
+    _check(lib.sp24_prune_2d(DTYPE_CODE[dt], M, K, _ptr(x), x.stride(0) if M > 1 else K, _ptr(out),
+                             out.stride(0) if M > 1 else K, _stream()), "sp24_prune_2d")
     return out

@@ -557,7 +557,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int cs = elem_bytes((sp24_dtype)p.cd_type);
     const int buf_bytes = 1024 * cs;
     const int nbuf = min(4, C::kEpiBytes / 4 / buf_bytes);  // staging buffers of this warp: 1, 2 or 4
-    const int ahead = nbuf >= 4 ? 2 : 1;            // boxes the C loads run ahead
+    const int ahead = nbuf > 1 ? nbuf - 1 : 1;      // boxes the C loads run ahead (their latency is what the epilogue waits on)
     // stores that may still be reading their buffer when the next buffer is claimed: with C the
     // buffer of box seq + ahead is claimed at the end of box seq, without C that of box seq + 1
     const int pending_ok = p.has_c ? nbuf - ahead : nbuf - 1;

@@ -30,84 +30,26 @@ __device__ __forceinline__ uint32_t mask_to_nibble(uint32_t mask) {
   return p0 | (p1 << 2);
 }
 
-// One group of four 16-bit values held in two words (lo = elements 0,1; hi = elements 2,3).
+// Which of a group's four 16-bit values (two words: lo = elements 0,1; hi = elements 2,3) are non-zero.
 struct Group16 {
-  static __device__ __forceinline__ uint32_t mask(uint32_t lo, uint32_t hi) {
-    return keep_mask4(lo & 0x7FFFu, (lo >> 16) & 0x7FFFu, hi & 0x7FFFu, (hi >> 16) & 0x7FFFu);
-  }
   static __device__ __forceinline__ uint32_t nonzero(uint32_t lo, uint32_t hi) {
     return ((lo & 0x7FFFu) != 0) | (((lo >> 16) & 0x7FFFu) != 0) << 1 | ((hi & 0x7FFFu) != 0) << 2 |
            (((hi >> 16) & 0x7FFFu) != 0) << 3;
   }
 };
 
-// One group of four int8 values in one word.  __vabs4 maps -128 to 0x80 = 128 (no saturation).
+// Which of a group's four int8 values (one word) are non-zero.
 struct Group8 {
-  static __device__ __forceinline__ uint32_t mask(uint32_t w) {
-    uint32_t a = __vabs4(w);
-    return keep_mask4(a & 0xFFu, (a >> 8) & 0xFFu, (a >> 16) & 0xFFu, a >> 24);
-  }
   static __device__ __forceinline__ uint32_t nonzero(uint32_t w) {
     return ((w & 0xFFu) != 0) | ((w & 0xFF00u) != 0) << 1 | ((w & 0xFF0000u) != 0) << 2 |
            ((w & 0xFF000000u) != 0) << 3;
   }
 };
 
-__device__ __forceinline__ uint32_t half_lane_mask(uint32_t keep2) {  // 2 keep bits -> 2x16-bit mask
-  return ((keep2 & 1u) ? 0x0000FFFFu : 0u) | ((keep2 & 2u) ? 0xFFFF0000u : 0u);
-}
-
-__device__ __forceinline__ uint32_t byte_lane_mask(uint32_t keep4) {  // 4 keep bits -> 4x8-bit mask
-  return ((keep4 & 1u) ? 0x000000FFu : 0u) | ((keep4 & 2u) ? 0x0000FF00u : 0u) |
-         ((keep4 & 4u) ? 0x00FF0000u : 0u) | ((keep4 & 8u) ? 0xFF000000u : 0u);
-}
-
 __device__ __forceinline__ uint4 ld_stream(const void* p) { return __ldcs(reinterpret_cast<const uint4*>(p)); }
 __device__ __forceinline__ void st_stream(void* p, uint4 v) { __stcs(reinterpret_cast<uint4*>(p), v); }
 
 // ---- prune -----------------------------------------------------------------------------
-template <int ES>
-__device__ __forceinline__ uint4 prune_vec(uint4 v) {
-  if (ES == 2) {
-    uint32_t m0 = Group16::mask(v.x, v.y), m1 = Group16::mask(v.z, v.w);
-    v.x &= half_lane_mask(m0);
-    v.y &= half_lane_mask(m0 >> 2);
-    v.z &= half_lane_mask(m1);
-    v.w &= half_lane_mask(m1 >> 2);
-  } else {
-    v.x &= byte_lane_mask(Group8::mask(v.x));
-    v.y &= byte_lane_mask(Group8::mask(v.y));
-    v.z &= byte_lane_mask(Group8::mask(v.z));
-    v.w &= byte_lane_mask(Group8::mask(v.w));
-  }
-  return v;
-}
-
-// Launch geometry of the vectorised kernels: blockDim = (TX, 256/TX), a warp always lies inside
-// one row; thread (tx, ty) of block (bx, by) handles units (bx*UNROLL + u)*TX + tx, u < UNROLL, of
-// rows by*TY + ty, + gridDim.y*TY, ...  No integer division on the device.
-// One 16-byte vector per thread and unroll step; `vpr` vectors per row.
-template <int ES, int UNROLL>
-__global__ void __launch_bounds__(kThreads) prune_vec_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
-                                                             uint8_t* y, int64_t row_bytes_y, int64_t vpr,
-                                                             int64_t rows) {
-  const int64_t c0 = (int64_t)blockIdx.x * UNROLL * blockDim.x + threadIdx.x;
-  for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows;
-       row += (int64_t)gridDim.y * blockDim.y) {
-    uint4 v[UNROLL];
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      int64_t c = c0 + (int64_t)u * blockDim.x;
-      if (c < vpr) v[u] = ld_stream(x + row * row_bytes_x + c * 16);
-    }
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      int64_t c = c0 + (int64_t)u * blockDim.x;
-      if (c < vpr) st_stream(y + row * row_bytes_y + c * 16, prune_vec<ES>(v[u]));
-    }
-  }
-}
-
 // Any alignment / leading dimension: one thread per group, element-wise accesses.
 template <typename T>
 __global__ void prune_scalar_kernel(const T* __restrict__ x, int64_t ldx, T* y, int64_t ldy, int64_t groups_per_row,
@@ -184,6 +126,73 @@ __device__ __forceinline__ uint32_t selection_index(uint32_t k_lo, uint32_t k_hi
   uint32_t r3 = (__byte_perm(k_lo, k_hi, 0x5410) | g) - __byte_perm(k_lo, k_hi, 0x7632);  // bit 15: c01, 31: c23
   uint32_t t = (r1 & g) | ((r2 & g) >> 1) | ((r3 & g) >> 2);    // bits 15..13: c02 c03 c01, 31..29: c13 c12 c23
   return ((t >> 13) & 7u) | ((t >> 26) & 0x38u);
+}
+
+// ---- prune (vectorised) -------------------------------------------------------------------------
+// Launch geometry of the vectorised kernels: blockDim = (TX, 256/TX), a warp always lies inside
+// one row; thread (tx, ty) of block (bx, by) handles units (bx*UNROLL + u)*TX + tx, u < UNROLL, of
+// rows by*TY + ty, + gridDim.y*TY, ...  No integer division on the device.
+//
+// Per comparison outcome the byte-permute selectors that copy the kept elements and zero the others
+// (selector nibble 4 = a zero byte of the second operand): 16-bit types need one selector for each
+// of the group's two words, int8 one for its single word.
+template <int ES>
+__device__ __forceinline__ uint32_t prune_selectors(uint32_t idx) {
+  const uint32_t mask = (selection_entry(idx) >> 4) & 0xFu;
+  if (ES == 2) {
+    uint32_t lo = ((mask & 1u) ? 0x10u : 0x44u) | (((mask & 2u) ? 0x32u : 0x44u) << 8);
+    uint32_t hi = ((mask & 4u) ? 0x10u : 0x44u) | (((mask & 8u) ? 0x32u : 0x44u) << 8);
+    return lo | (hi << 16);
+  }
+  return ((mask & 1u) ? 0x0u : 0x4u) | (((mask & 2u) ? 0x1u : 0x4u) << 4) | (((mask & 4u) ? 0x2u : 0x4u) << 8) |
+         (((mask & 8u) ? 0x3u : 0x4u) << 12);
+}
+
+template <int ES>
+__device__ __forceinline__ uint4 prune_vec(uint4 v, const uint32_t* table) {
+  if (ES == 2) {
+    const uint32_t s0 = table[selection_index(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu)];
+    const uint32_t s1 = table[selection_index(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu)];
+    return make_uint4(__byte_perm(v.x, 0, s0 & 0xFFFFu), __byte_perm(v.y, 0, s0 >> 16), __byte_perm(v.z, 0, s1 & 0xFFFFu),
+                      __byte_perm(v.w, 0, s1 >> 16));
+  }
+  uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    const uint32_t a = __vabs4(w[g]);  // -128 -> 0x80 = 128, no saturation
+    w[g] = __byte_perm(w[g], 0, table[selection_index(__byte_perm(a, 0, 0x4140), __byte_perm(a, 0, 0x4342))]);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// One 16-byte vector per thread and unroll step; `vpr` vectors per row.
+template <int ES, int UNROLL>
+__global__ void __launch_bounds__(kThreads) prune_vec_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
+                                                             uint8_t* y, int64_t row_bytes_y, int64_t vpr,
+                                                             int64_t rows) {
+  __shared__ uint32_t table[64];
+  {
+    const int t = threadIdx.y * blockDim.x + threadIdx.x;
+    if (t < 64) table[t] = prune_selectors<ES>((uint32_t)t);
+    __syncthreads();
+  }
+  const uint32_t c0 = blockIdx.x * UNROLL * blockDim.x + threadIdx.x;
+  for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows;
+       row += (int64_t)gridDim.y * blockDim.y) {
+    const uint8_t* xr = x + row * row_bytes_x;
+    uint8_t* yr = y + row * row_bytes_y;
+    uint4 v[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const uint32_t c = c0 + u * blockDim.x;
+      if (c < vpr) v[u] = ld_stream(xr + c * 16u);
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const uint32_t c = c0 + u * blockDim.x;
+      if (c < vpr) st_stream(yr + c * 16u, prune_vec<ES>(v[u], table));
+    }
+  }
 }
 
 template <bool COUNT>

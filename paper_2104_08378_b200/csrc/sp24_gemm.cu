@@ -106,7 +106,6 @@ struct Shared {
   uint64_t c_full[4][4];           // per epilogue warp and staging buffer: C box has landed
   uint32_t tmem_base;
   volatile uint32_t abort;
-  volatile uint32_t c_hint_tiles;  // tiles whose main loop is close enough to its end to fetch C into the L2
 };
 static_assert(sizeof(Shared) <= 512, "barrier block");
 
@@ -368,7 +367,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     for (int w = 0; w < 4; ++w)
       for (int b = 0; b < 4; ++b) ptx::mbar_init(&sh->c_full[w][b], 1);
     sh->abort = 0;
-    sh->c_hint_tiles = 0;
     if (blockIdx.x == 0) p.status[0] = 0;  // a wait can only expire a second later
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&map_a);
@@ -391,11 +389,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     // ------------------------------ TMA producer ------------------------------
     if (ptx::elect_one()) {
       int stage = 0;
-      uint32_t phase = 0, tiles_started = 0;
+      uint32_t phase = 0;
       const int box_elems = C::kAtomElems;  // elements per 128-byte atom row
-      const int hint_kb = max(0, p.k_blocks - 24);  // when the epilogue warps should pull C into the L2
       for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
-        ++tiles_started;
         int mt, nt;
         tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
         // the last n-tile may be narrower: the pair then splits only the columns that exist
@@ -415,7 +411,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!bounded_wait(&sh->empty[stage], phase ^ 1u, sh, p.status, 1u)) break;
-          if (kb == hint_kb) sh->c_hint_tiles = tiles_started;
           uint8_t* sa = smem + stage * C::kStageBytes;
           uint8_t* sb = sa + C::kABytes;
           uint8_t* se = sb + C::kBBytes;
@@ -596,19 +591,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       for (int i = 0; i < ahead; ++i) issue_c_load();
 
     int acc = 0;
-    uint32_t acc_phase = 0, seq = 0, tiles_seen = 0;
+    uint32_t acc_phase = 0, seq = 0;
     for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
-      ++tiles_seen;
-      if (p.has_c && lane == 0) {
-        // Shortly before the main loop ends, ask the L2 for this warp's boxes of C so that the loads
-        // above are L2 hits.  The wait is only a hint and gives up after a while.
-        for (uint32_t spin = 0; sh->c_hint_tiles < tiles_seen && spin < (1u << 20) && !sh->abort; ++spin) __nanosleep(128);
-        for (int it = 0; it < kIters; ++it) {
-          int row0, col0;
-          if (box_of(t, it, row0, col0))
-            ptx::tma_prefetch_2d(&map_c, p.cd_col_major ? row0 : col0, p.cd_col_major ? col0 : row0);
-        }
-      }
       if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u)) break;
       ptx::tc_fence_after();
       uint32_t r_next[32];

@@ -560,23 +560,27 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     constexpr int kSub = BLOCK_N / 32;
     constexpr int kIters = MBLK * kSub;
 
-    // box `it` of tile `t`: first row / column and whether any of it lies inside the matrix
-    auto box_of = [&](int t, int it, int& row0, int& col0) -> bool {
-      int mt, nt;
-      tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
+    // box `it` of the tile (mt, nt): first row / column and whether any of it lies inside the matrix
+    auto box_of = [&](int mt, int nt, int it, int& row0, int& col0) -> bool {
       const int j = it / kSub, sc = it - j * kSub;
       row0 = ((mt * MBLK + j) * CTAS + (int)cta_rank) * kBlockM + q * 32;
       col0 = nt * BLOCK_N + sc * 32;
       return row0 < p.M && col0 < p.N;
     };
     // cursor of the C loads over the same stream of boxes, `ahead` live boxes in front of the consumer
-    int pf_t = cluster_id, pf_it = 0;
+    // (the tile coordinates cost two divisions: once per tile, not per box)
+    int pf_t = cluster_id, pf_it = 0, pf_mt = 0, pf_nt = 0;
+    if (pf_t < num_tiles) tile_coords(pf_t, p.m_tiles, p.n_tiles, p.band, pf_mt, pf_nt);
     uint32_t pf_seq = 0;
     auto issue_c_load = [&]() {  // lane 0 only: load the next live box of the stream, if any
       while (pf_t < num_tiles) {
         int row0, col0;
-        const bool live_box = box_of(pf_t, pf_it, row0, col0);
-        if (++pf_it == kIters) { pf_it = 0; pf_t += num_clusters; }
+        const bool live_box = box_of(pf_mt, pf_nt, pf_it, row0, col0);
+        if (++pf_it == kIters) {
+          pf_it = 0;
+          pf_t += num_clusters;
+          if (pf_t < num_tiles) tile_coords(pf_t, p.m_tiles, p.n_tiles, p.band, pf_mt, pf_nt);
+        }
         if (live_box) {
           const int b = pf_seq % nbuf;
           ptx::mbar_expect_tx(&sh->c_full[q][b], (uint32_t)buf_bytes);
@@ -593,6 +597,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     int acc = 0;
     uint32_t acc_phase = 0, seq = 0;
     for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
+      int mt, nt;
+      tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
       if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u)) break;
       ptx::tc_fence_after();
       uint32_t r_next[32];
@@ -610,7 +616,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           ptx::tmem_ld_32x32b_x32(t_acc + jn * BLOCK_N + scn * 32, r_next);
         }
         int row0, col0;
-        if (!box_of(t, it, row0, col0)) continue;  // same answer for the whole warp
+        if (!box_of(mt, nt, it, row0, col0)) continue;  // same answer for the whole warp
         const int b = seq % nbuf;
         uint8_t* buf = my_bufs + b * buf_bytes;
         if (p.has_c && !bounded_wait(&sh->c_full[q][b], (seq / nbuf) & 1u, sh, p.status, 5u)) { ok = false; break; }

@@ -36,7 +36,8 @@ namespace {
 
 constexpr int kBlockM = 128;              // rows of A per CTA and m-block (tensor-memory lanes)
 constexpr int kAtomBytes = 128;           // bytes per row of one swizzle-128B operand atom
-constexpr int kNumThreads = 192;          // 6 warps
+constexpr int kEpiWarps = 8;              // two per tensor-memory lane quarter, taking alternate boxes
+constexpr int kNumThreads = 64 + 32 * kEpiWarps;  // TMA producer, MMA issuer, epilogue warps
 constexpr long long kWaitTimeoutCycles = 2000ll * 1000ll * 1000ll;  // per wait: 1-2 s of SM clock
 constexpr uint32_t kTmemCols = 512;
 
@@ -103,7 +104,7 @@ struct Cfg {
 
 struct Shared {
   uint64_t full[8], empty[8], tmem_full[2], tmem_empty[2];
-  uint64_t c_full[4][4];           // per epilogue warp and staging buffer: C box has landed
+  uint64_t c_full[kEpiWarps][4];   // per epilogue warp and staging buffer: C box has landed
   uint32_t tmem_base;
   volatile uint32_t abort;
 };
@@ -362,9 +363,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(&sh->tmem_full[a], 1);
-      ptx::mbar_init(&sh->tmem_empty[a], 4 * CTAS);  // one arrival per epilogue warp of the pair
+      ptx::mbar_init(&sh->tmem_empty[a], kEpiWarps * CTAS);  // one arrival per epilogue warp of the pair
     }
-    for (int w = 0; w < 4; ++w)
+    for (int w = 0; w < kEpiWarps; ++w)
       for (int b = 0; b < 4; ++b) ptx::mbar_init(&sh->c_full[w][b], 1);
     sh->abort = 0;
     if (blockIdx.x == 0) p.status[0] = 0;  // a wait can only expire a second later
@@ -549,14 +550,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     // (if beta != 0) into a staging buffer a few boxes ahead, tcgen05.ld of the accumulator columns,
     // convert in place, TMA store of the D box.  Boxes outside the matrix are clipped by the TMA.
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+    const int ew = warp - 2;  // epilogue warp 0..7: warps ew and ew + 4 share a lane quarter
     const int cs = elem_bytes((sp24_dtype)p.cd_type);
     const int buf_bytes = 1024 * cs;
-    const int nbuf = min(4, C::kEpiBytes / 4 / buf_bytes);  // staging buffers of this warp: 1, 2 or 4
+    // Both warps of a quarter work (alternate boxes) when each can have a staging buffer of its own;
+    // otherwise the second one only takes part in handing the accumulators back.
+    const int split = (C::kEpiBytes / kEpiWarps >= buf_bytes) ? 2 : 1;
+    const int first_it = ew >> 2;
+    const bool active = first_it < split;
+    const int warp_bytes = C::kEpiBytes / (4 * split);
+    const int nbuf = min(4, warp_bytes / buf_bytes);  // staging buffers of this warp: 1, 2 or 4
     const int ahead = nbuf > 1 ? nbuf - 1 : 1;      // boxes the C loads run ahead (their latency is what the epilogue waits on)
     // stores that may still be reading their buffer when the next buffer is claimed: with C the
     // buffer of box seq + ahead is claimed at the end of box seq, without C that of box seq + 1
     const int pending_ok = p.has_c ? nbuf - ahead : nbuf - 1;
-    uint8_t* my_bufs = epi + q * (C::kEpiBytes / 4);
+    uint8_t* my_bufs = epi + (ew & (4 * split - 1)) * warp_bytes;
     constexpr int kSub = BLOCK_N / 32;
     constexpr int kIters = MBLK * kSub;
 
@@ -569,29 +577,30 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     };
     // cursor of the C loads over the same stream of boxes, `ahead` live boxes in front of the consumer
     // (the tile coordinates cost two divisions: once per tile, not per box)
-    int pf_t = cluster_id, pf_it = 0, pf_mt = 0, pf_nt = 0;
+    int pf_t = cluster_id, pf_it = first_it, pf_mt = 0, pf_nt = 0;
     if (pf_t < num_tiles) tile_coords(pf_t, p.m_tiles, p.n_tiles, p.band, pf_mt, pf_nt);
     uint32_t pf_seq = 0;
     auto issue_c_load = [&]() {  // lane 0 only: load the next live box of the stream, if any
       while (pf_t < num_tiles) {
         int row0, col0;
         const bool live_box = box_of(pf_mt, pf_nt, pf_it, row0, col0);
-        if (++pf_it == kIters) {
-          pf_it = 0;
+        pf_it += split;
+        if (pf_it >= kIters) {
+          pf_it = first_it;
           pf_t += num_clusters;
           if (pf_t < num_tiles) tile_coords(pf_t, p.m_tiles, p.n_tiles, p.band, pf_mt, pf_nt);
         }
         if (live_box) {
           const int b = pf_seq % nbuf;
-          ptx::mbar_expect_tx(&sh->c_full[q][b], (uint32_t)buf_bytes);
-          ptx::tma_load_2d(my_bufs + b * buf_bytes, &map_c, &sh->c_full[q][b], p.cd_col_major ? row0 : col0,
+          ptx::mbar_expect_tx(&sh->c_full[ew][b], (uint32_t)buf_bytes);
+          ptx::tma_load_2d(my_bufs + b * buf_bytes, &map_c, &sh->c_full[ew][b], p.cd_col_major ? row0 : col0,
                            p.cd_col_major ? col0 : row0);
           ++pf_seq;
           return;
         }
       }
     };
-    if (p.has_c && lane == 0)
+    if (p.has_c && active && lane == 0)
       for (int i = 0; i < ahead; ++i) issue_c_load();
 
     int acc = 0;
@@ -603,23 +612,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       ptx::tc_fence_after();
       uint32_t r_next[32];
       const uint32_t t_acc = tmem_base + (acc * MBLK) * BLOCK_N + ((uint32_t)(q * 32) << 16);
-      ptx::tmem_ld_32x32b_x32(t_acc, r_next);
+      if (active) {
+        const int j0 = first_it / kSub, sc0 = first_it - j0 * kSub;
+        ptx::tmem_ld_32x32b_x32(t_acc + j0 * BLOCK_N + sc0 * 32, r_next);
+      }
       bool ok = true;
 #pragma unroll 1
-      for (int it = 0; it < kIters; ++it) {
+      for (int it = active ? first_it : kIters; it < kIters; it += split) {
         uint32_t r[32];
         ptx::tmem_ld_wait();
 #pragma unroll
         for (int e = 0; e < 32; ++e) r[e] = r_next[e];
-        if (it + 1 < kIters) {
-          const int jn = (it + 1) / kSub, scn = (it + 1) - jn * kSub;
+        if (it + split < kIters) {
+          const int jn = (it + split) / kSub, scn = (it + split) - jn * kSub;
           ptx::tmem_ld_32x32b_x32(t_acc + jn * BLOCK_N + scn * 32, r_next);
         }
         int row0, col0;
         if (!box_of(mt, nt, it, row0, col0)) continue;  // same answer for the whole warp
         const int b = seq % nbuf;
         uint8_t* buf = my_bufs + b * buf_bytes;
-        if (p.has_c && !bounded_wait(&sh->c_full[q][b], (seq / nbuf) & 1u, sh, p.status, 5u)) { ok = false; break; }
+        if (p.has_c && !bounded_wait(&sh->c_full[ew][b], (seq / nbuf) & 1u, sh, p.status, 5u)) { ok = false; break; }
         if (KIND == 1 && p.dequant) {
           // this thread's output row: its scale and bias
           const int row = min(row0 + lane, (int)p.M - 1);

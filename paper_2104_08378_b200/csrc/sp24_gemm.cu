@@ -9,8 +9,9 @@
 //            memory (tcgen05.cp), issues the tcgen05.mma[.sp] of the stage, commits the stage
 //            back to the producer and, after the last k-block, the accumulators to the epilogue;
 //            owns the tensor-memory allocation;
-//   warps 2-5 epilogue: tcgen05.ld accumulator -> registers, alpha/beta, convert, store; the loads
-//            of C and of the next accumulator chunk run one chunk ahead.
+//   warps 2-9 epilogue, two per tensor-memory lane quarter taking alternate 32-column boxes:
+//            tcgen05.ld accumulator -> registers, alpha/beta, convert into a staging buffer, TMA
+//            store; the TMA loads of C run a few boxes ahead, the next tcgen05.ld one box ahead.
 // CTAS == 2 runs a pair of CTAs (cluster of two): each CTA loads its 128 rows of A / metadata per
 // m-block and its half of B, CTA 0 issues cta_group::2 MMAs (M = 256) for both.
 // MBLK == 2 gives every CTA two m-blocks (two accumulators, one B tile): what an SM can pull in

@@ -55,8 +55,13 @@ typedef enum {
 
 /* SP24_F32 as an OPERAND type selects the TF32 mode (Section 3.2, Table 1): FP32 storage, TF32
  * multiplication, FP32 accumulation, and the 1:2 pattern -- one kept value in every aligned
- * PAIR along K instead of two in every group of four. */
-typedef enum { SP24_F16 = 0, SP24_BF16 = 1, SP24_I8 = 2, SP24_F32 = 3, SP24_I32 = 4 } sp24_dtype;
+ * PAIR along K instead of two in every group of four.
+ * SP24_E4M3 / SP24_E5M2 are the 8-bit floating-point encodings (1-4-3 without infinities, and
+ * 1-5-2).  Table 1 of the paper has no 8-bit floating-point row (its hardware had none); they
+ * use the 2:4 pattern and the format of the 8-bit integer row, with FP32 accumulation. */
+typedef enum {
+  SP24_F16 = 0, SP24_BF16 = 1, SP24_I8 = 2, SP24_F32 = 3, SP24_I32 = 4, SP24_E4M3 = 5, SP24_E5M2 = 6
+} sp24_dtype;
 
 /* Metadata layouts.
  * CANONICAL: row i occupies K/8 bytes starting at meta + i*K/8; group g of the row (columns
@@ -92,8 +97,9 @@ size_t sp24_meta_bytes(sp24_dtype t, int64_t M, int64_t K, sp24_meta_layout l);
  * For every row i < M and every aligned group of four columns 4g..4g+3 < K the two values of
  * largest magnitude are copied bit-for-bit to y, the other two positions receive +0.  Equal
  * magnitudes: the lower column index is kept.  Magnitude is |x| for I8 (so -128 ranks as
- * 128) and the bit pattern without its sign bit for F16/BF16 (denormals are not flushed).
- *   t: SP24_F16, SP24_BF16 or SP24_I8.      M >= 0, K >= 0, K % 4 == 0.
+ * 128) and the bit pattern without its sign bit for F16/BF16/E4M3/E5M2 (denormals are not
+ * flushed).
+ *   t: SP24_F16, SP24_BF16, SP24_I8, SP24_E4M3 or SP24_E5M2.   M >= 0, K >= 0, K % 4 == 0.
  *      SP24_F32: the 1:2 pattern -- the larger magnitude of every aligned pair is kept, equal
  *      magnitudes keep the first (K % 8 == 0, 16-byte aligned pointers and rows required;
  *      the same holds for sp24_compress / sp24_decompress, whose vals are then M x K/2 FP32).
@@ -129,11 +135,14 @@ sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals
  *   ab_type: SP24_F16 or SP24_BF16 (FP32 accumulate), SP24_I8 (INT32 accumulate) or SP24_F32
  *            (TF32 mode, 1:2 pattern, FP32 accumulate; cd_type SP24_F32 and K-contiguous B
  *            only; inputs are used with their low 13 mantissa bits ignored) -- the
- *            operand/accumulator pairs of Table 1.
+ *            operand/accumulator pairs of Table 1.  SP24_E4M3 or SP24_E5M2 (both operands the
+ *            same type, FP32 accumulate, K-contiguous B only) go beyond that table.
  *   cd_type: type of C and D.  F16/BF16 operands: SP24_F16, SP24_BF16 (ab_type's own) or
- *            SP24_F32.  I8 operands: SP24_I32.
+ *            SP24_F32.  I8 operands: SP24_I32.  E4M3/E5M2 operands: SP24_F16, SP24_BF16 or
+ *            SP24_F32.
  *   M, N, K: K is the LOGICAL (uncompressed) reduction length.  M, N, K must be multiples of
- *            16 (16-bit types) or 32 (I8) (Section 3.2); zero-sized problems return SP24_OK.
+ *            16 (16-bit types) or 32 (8-bit types) (Section 3.2); zero-sized problems return
+ *            SP24_OK.
  *   lda:     leading dimension of the A-side value array: of vals (M x K/2) when
  *            a_is_dense == 0, of the dense M x K matrix when a_is_dense == 1.
  *   order_b: SP24_COL_MAJOR = K contiguous (B stored as N rows of K values: the
@@ -159,7 +168,7 @@ size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d);
 
 /* The 2:4 sparse GEMM on the sparse tensor cores (Section 3.2, Figure 2):
  *   D[i,j] = alpha * sum_g sum_{t=0,1} vals[i,2g+t] * B[4g + p_t(i,g), j] + beta * C[i,j].
- *   alpha, beta: HOST pointers.  float for F16/BF16 operands; int32_t for I8, where only
+ *   alpha, beta: HOST pointers.  float for floating-point operands; int32_t for I8, where only
  *                alpha == 1 and beta in {0, 1} are built (else SP24_ERR_UNSUPPORTED).
  *   A:    device; vals (M x K/2) or dense A (M x K), row-major, 16-byte aligned.
  *   meta: device; TCGEN05-layout metadata of A (ignored when a_is_dense).
@@ -230,7 +239,8 @@ sp24_status sp24_gemm_static_ws(const sp24_gemm_desc* d, const void* alpha, cons
 /* Lowering of a 3x3, stride-1, pad-1 NHWC convolution input to the GEMM's B operand
  * (Section 4.2: a convolution's reduction dimension is C*R*S).  Output is K-contiguous:
  *   out[((n*H + h)*W + w) * ldo + (r*3 + s)*C + c] = in[n, h+r-1, w+s-1, c]  (0 outside).
- *   t: SP24_F16, SP24_BF16 or SP24_I8.  C*sizeof(t) must be a multiple of 16; ldo >= 9*C. */
+ *   t: SP24_F16, SP24_BF16, SP24_I8, SP24_E4M3 or SP24_E5M2.  C*sizeof(t) must be a multiple
+ *   of 16; ldo >= 9*C. */
 sp24_status sp24_im2col_nhwc_3x3(sp24_dtype t, int64_t Nb, int64_t H, int64_t W, int64_t C,
                                  const void* in, void* out, int64_t ldo, void* stream);
 

@@ -5,7 +5,8 @@ C, fp64 / int64 arithmetic).  It imports nothing from the CUDA package and the C
 imports nothing from here.  Callers: the tests, the smoke check and the bench's CPU legs.
 
 Array conventions: fp16 and bf16 matrices travel as ``numpy.uint16`` BIT PATTERNS, int8 as
-``numpy.int8``; ``dtype`` is one of the strings "f16", "bf16", "i8".  All matrices are 2-D,
+``numpy.int8``, the 8-bit floats as ``numpy.uint8`` bit patterns; ``dtype`` is one of the strings
+"f16", "bf16", "i8", "e4m3", "e5m2".  All matrices are 2-D,
 C-contiguous (row-major).  B is passed as an ``N x K`` array (K contiguous), i.e. the
 transpose of the K x N matrix of Section 3.2.
 """
@@ -21,7 +22,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "sp24_oracle.c")
 _LIB = os.path.join(_HERE, "libsp24_oracle.so")
 
-DTYPE_CODE = {"f16": 0, "bf16": 1, "i8": 2}
+DTYPE_CODE = {"f16": 0, "bf16": 1, "i8": 2, "e4m3": 5, "e5m2": 6}
 C_DTYPE_CODE = {"f16": 0, "bf16": 1, "f32": 3, "i32": 4}
 
 
@@ -84,6 +85,8 @@ def _load():
         lib.oracle_prune_2d.restype = None
         lib.oracle_dequant.argtypes = [i64, i64, vp, vp, vp, i32, ctypes.c_float, vp, vp]
         lib.oracle_dequant.restype = None
+        lib.oracle_to_double.argtypes = [i32, i64, vp, vp]
+        lib.oracle_to_double.restype = None
         lib.oracle_im2col_nhwc_3x3.argtypes = [i32, i64, i64, i64, i64, vp, vp, i64]
         lib.oracle_im2col_nhwc_3x3.restype = None
         _lib = lib
@@ -95,7 +98,7 @@ def num_threads() -> int:
 
 
 def _np_elem(dtype: str):
-    return np.int8 if dtype == "i8" else np.uint16
+    return np.int8 if dtype == "i8" else (np.uint8 if dtype in ("e4m3", "e5m2") else np.uint16)
 
 
 def _check(a: np.ndarray, dtype: str, name: str) -> np.ndarray:
@@ -349,4 +352,9 @@ def bits_to_float64(a: np.ndarray, dtype: str) -> np.ndarray:
         return a.astype(np.float64)
     if dtype == "f16":
         return a.view(np.float16).astype(np.float64)
+    if dtype in ("e4m3", "e5m2"):
+        a = np.ascontiguousarray(a)
+        out = np.empty(a.shape, dtype=np.float64)
+        _load().oracle_to_double(DTYPE_CODE[dtype], a.size, _ptr(a), _ptr(out))
+        return out
     return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)

@@ -11,8 +11,9 @@
  * double; the int8 GEMM accumulates in int64.  The only concession to run time is an OpenMP
  * "parallel for" over output rows (rows are independent in every operation here).
  *
- * dtype codes: 0 = fp16, 1 = bf16, 2 = int8.  Matrices are row-major with a leading
- * dimension in elements unless stated.
+ * dtype codes: 0 = fp16, 1 = bf16, 2 = int8, 5 = fp8 e4m3, 6 = fp8 e5m2 (the 8-bit floating-point
+ * types are not in the paper: same 2:4 pattern and format, OCP 8-bit floating-point encodings).
+ * Matrices are row-major with a leading dimension in elements unless stated.
  *
  * Pins (tests/test_oracle_*.py): the pattern invariant and idempotence, brute force over all
  * C(4,2) keep-patterns, the metadata example of Section 3.1, the storage arithmetic of
@@ -32,7 +33,8 @@
 /* element helpers                                                                       */
 /* ------------------------------------------------------------------------------------- */
 
-static int elem_size(int dtype) { return dtype == 2 ? 1 : 2; }
+static int elem_size(int dtype) { return (dtype == 2 || dtype == 5 || dtype == 6) ? 1 : 2; }
+static int is_fp8(int dtype) { return dtype == 5 || dtype == 6; }
 
 /* IEEE binary16 bit pattern -> double, exactly. */
 static double half_bits_to_double(uint16_t h) {
@@ -58,7 +60,35 @@ static double bf16_bits_to_double(uint16_t b) {
   return (double)f;
 }
 
+/* 8-bit floating point, e4m3: 1 sign, 4 exponent (bias 7), 3 mantissa bits; no infinities, the
+ * single NaN pattern per sign is exponent and mantissa all ones; largest finite value 448. */
+static double e4m3_bits_to_double(uint8_t b) {
+  int sign = (b >> 7) & 1;
+  int exponent = (b >> 3) & 0xF;
+  int mantissa = b & 0x7;
+  double v;
+  if (exponent == 15 && mantissa == 7) v = NAN;
+  else if (exponent == 0) v = ldexp((double)mantissa, -9); /* m/8 * 2^-6 */
+  else v = ldexp((double)(mantissa + 8), exponent - 10);   /* (1 + m/8) * 2^(e-7) */
+  return sign ? -v : v;
+}
+
+/* 8-bit floating point, e5m2: 1 sign, 5 exponent (bias 15), 2 mantissa bits; IEEE-style
+ * infinities and NaNs. */
+static double e5m2_bits_to_double(uint8_t b) {
+  int sign = (b >> 7) & 1;
+  int exponent = (b >> 2) & 0x1F;
+  int mantissa = b & 0x3;
+  double v;
+  if (exponent == 31) v = mantissa ? NAN : INFINITY;
+  else if (exponent == 0) v = ldexp((double)mantissa, -16); /* m/4 * 2^-14 */
+  else v = ldexp((double)(mantissa + 4), exponent - 17);    /* (1 + m/4) * 2^(e-15) */
+  return sign ? -v : v;
+}
+
 static double load_as_double(int dtype, const void* base, int64_t index) {
+  if (dtype == 5) return e4m3_bits_to_double(((const uint8_t*)base)[index]);
+  if (dtype == 6) return e5m2_bits_to_double(((const uint8_t*)base)[index]);
   if (dtype == 0) return half_bits_to_double(((const uint16_t*)base)[index]);
   if (dtype == 1) return bf16_bits_to_double(((const uint16_t*)base)[index]);
   return (double)((const int8_t*)base)[index];
@@ -66,8 +96,10 @@ static double load_as_double(int dtype, const void* base, int64_t index) {
 
 /* Magnitude key used by the pruning criterion (Section 4.1, step 2).
  * 16-bit floats: the bit pattern without the sign bit, which orders finite values by |x|
- * (zero of either sign -> 0, subnormals keep their rank).  int8: |x| as an int, -128 -> 128. */
+ * (zero of either sign -> 0, subnormals keep their rank).  int8: |x| as an int, -128 -> 128.
+ * 8-bit floats: the seven bits below the sign, same argument as for the 16-bit floats. */
 static int magnitude_key(int dtype, const void* base, int64_t index) {
+  if (is_fp8(dtype)) return ((const uint8_t*)base)[index] & 0x7F;
   if (dtype == 2) {
     int v = ((const int8_t*)base)[index];
     return v < 0 ? -v : v;
@@ -96,12 +128,12 @@ static void select_two(const int key[4], int* p0, int* p1) {
 }
 
 static void copy_elem(int dtype, void* dst, int64_t di, const void* src, int64_t si) {
-  if (dtype == 2) ((int8_t*)dst)[di] = ((const int8_t*)src)[si];
+  if (elem_size(dtype) == 1) ((int8_t*)dst)[di] = ((const int8_t*)src)[si];
   else ((uint16_t*)dst)[di] = ((const uint16_t*)src)[si];
 }
 
 static void zero_elem(int dtype, void* dst, int64_t di) {
-  if (dtype == 2) ((int8_t*)dst)[di] = 0;
+  if (elem_size(dtype) == 1) ((int8_t*)dst)[di] = 0;
   else ((uint16_t*)dst)[di] = 0; /* +0 */
 }
 
@@ -199,7 +231,7 @@ void oracle_decompress(int dtype, int64_t M, int64_t K, const void* vals, int64_
 /* direction 0: canonical -> operand order, 1: operand order -> canonical.                 */
 /* ------------------------------------------------------------------------------------- */
 static int64_t operand_bit_in_block(int dtype, int r, int q) {
-  if (dtype == 2) return 128 * (int64_t)r + 4 * q;
+  if (elem_size(dtype) == 1) return 128 * (int64_t)r + 4 * q;
   return 128 * (r % 8) + 16 * ((r / 8) % 2) + 2048 * (r / 16) + 1024 * ((q / 4) % 2) +
          32 * (q / 8) + 4 * (q % 4);
 }
@@ -593,3 +625,8 @@ void oracle_prune_2d(int dtype, int64_t M, int64_t K, const void* x, int64_t ldx
 }
 
 int oracle_elem_size(int dtype) { return elem_size(dtype); }
+
+/* Exact widening of n stored elements to double. */
+void oracle_to_double(int dtype, int64_t n, const void* x, double* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = load_as_double(dtype, x, i);
+}

@@ -18,14 +18,14 @@ import torch
 from .build import LIB_PATH
 
 OK = 0
-F16, BF16, I8, F32, I32 = 0, 1, 2, 3, 4
+F16, BF16, I8, F32, I32, E4M3, E5M2 = 0, 1, 2, 3, 4, 5, 6
 META_CANONICAL, META_TCGEN05 = 0, 1
 ROW_MAJOR, COL_MAJOR = 0, 1
-DTYPE_CODE = {"f16": F16, "bf16": BF16, "i8": I8, "f32": F32, "i32": I32}
+DTYPE_CODE = {"f16": F16, "bf16": BF16, "i8": I8, "f32": F32, "i32": I32, "e4m3": E4M3, "e5m2": E5M2}
 TORCH_DTYPE = {"f16": torch.float16, "bf16": torch.bfloat16, "i8": torch.int8, "f32": torch.float32,
-               "i32": torch.int32}
+               "i32": torch.int32, "e4m3": torch.float8_e4m3fn, "e5m2": torch.float8_e5m2}
 _FROM_TORCH = {torch.float16: "f16", torch.bfloat16: "bf16", torch.int8: "i8", torch.float32: "f32",
-               torch.int32: "i32"}
+               torch.int32: "i32", torch.float8_e4m3fn: "e4m3", torch.float8_e5m2: "e5m2"}
 
 EXPORTS = [
     "sp24_status_string", "sp24_values_bytes", "sp24_meta_bytes", "sp24_prune", "sp24_compress",
@@ -199,7 +199,7 @@ def gemm(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor, *, alpha=
     K = A.shape[1] if a_is_dense else 2 * A.shape[1]
     N = Bt.shape[1] if b_row_major else Bt.shape[0]
     assert (Bt.shape[0] if b_row_major else Bt.shape[1]) == K
-    cd = cd or ("i32" if ab == "i8" else ab)
+    cd = cd or ("i32" if ab == "i8" else ("bf16" if ab in ("e4m3", "e5m2") else ab))
     if out is None:
         out = torch.empty((N, M) if cd_col_major else (M, N), dtype=TORCH_DTYPE[cd], device=A.device)
     ws = ws if ws is not None else workspace(A.device)
@@ -235,7 +235,7 @@ def gemm_static_ws(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor,
     M = A.shape[0]
     K = A.shape[1] if a_is_dense else 2 * A.shape[1]
     N = Bt.shape[0]
-    cd = cd or ("i32" if ab == "i8" else ab)
+    cd = cd or ("i32" if ab == "i8" else ("bf16" if ab in ("e4m3", "e5m2") else ab))
     desc = make_desc(ab, cd, M, N, K, A.stride(0), Bt.stride(0), C.stride(0) if C is not None else N,
                      out.stride(0), a_is_dense)
     a, b = _scalar(ab, alpha), _scalar(ab, beta)
@@ -272,7 +272,7 @@ def conv3x3_nhwc(A: torch.Tensor, meta: torch.Tensor | None, x: torch.Tensor, *,
     Nb, H, W, Cin = x.shape
     M = A.shape[0]
     K, N = 9 * Cin, Nb * H * W
-    cd = cd or ("i32" if ab == "i8" else ab)
+    cd = cd or ("i32" if ab == "i8" else ("bf16" if ab in ("e4m3", "e5m2") else ab))
     if out is None:
         out = torch.empty((N, M) if nhwc_out else (M, N), dtype=TORCH_DTYPE[cd], device=A.device)
     ws = ws if ws is not None else workspace(A.device)

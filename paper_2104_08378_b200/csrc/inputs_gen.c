@@ -6,7 +6,8 @@
  * kinds: 0 = N(0, p0) by Box-Muller, 1 = U(p0, p1), 2 = integers uniform in [-127, 127],
  *        3 = max(N(0, p0), 0).
  * dtype: 0 = fp16 bits, 1 = bf16 bits (both round-to-nearest-even), 2 = int8,
- *        3 = fp32 bits holding a TF32-representable value (10 mantissa bits, round-to-nearest-even).
+ *        3 = fp32 bits holding a TF32-representable value (10 mantissa bits, round-to-nearest-even),
+ *        5 = fp8 e4m3 bits, 6 = fp8 e5m2 bits (round-to-nearest-even, saturating at the largest finite value).
  */
 #include <math.h>
 #include <stdint.h>
@@ -55,6 +56,33 @@ static uint16_t double_to_half_rne(double d) {
   return bits;
 }
 
+/* 8-bit float with `mbits` mantissa bits and exponent bias `bias`; `max_bits` is the pattern of
+ * the largest finite magnitude (results beyond it saturate there). */
+static uint8_t double_to_fp8_rne(double d, int mbits, int bias, int max_bits) {
+  uint8_t sign = signbit(d) ? 0x80 : 0;
+  double a = fabs(d);
+  int bits;
+  if (a != a) return (uint8_t)(sign | 0x7F);
+  if (a == 0.0) return sign;
+  int e;
+  frexp(a, &e); /* a = f * 2^e, f in [0.5, 1): unbiased exponent e - 1 */
+  int E = e - 1;
+  if (E < 1 - bias) {
+    /* subnormal range: units of 2^(1 - bias - mbits); a carry into the first normal is the right pattern */
+    bits = (int)rint(ldexp(a, -(1 - bias - mbits)));
+  } else {
+    int q = (int)rint(ldexp(a, mbits - E)); /* in [2^mbits, 2^(mbits+1)] */
+    if (q == (2 << mbits)) { q >>= 1; ++E; }
+    bits = ((E + bias) << mbits) | (q - (1 << mbits));
+  }
+  if (bits > max_bits) bits = max_bits;
+  return (uint8_t)(sign | bits);
+}
+
+uint8_t sp24_inputs_to_fp8(double d, int e5m2) {
+  return e5m2 ? double_to_fp8_rne(d, 2, 15, 0x7B) : double_to_fp8_rne(d, 3, 7, 0x7E);
+}
+
 void sp24_inputs_fill(int kind, double p0, double p1, int dtype, uint64_t seed,
                       uint64_t tensor_id, uint64_t start, uint64_t count, void* out) {
   const uint64_t k0 = stream_key(seed, tensor_id, 0), k1 = stream_key(seed, tensor_id, 1);
@@ -72,7 +100,8 @@ void sp24_inputs_fill(int kind, double p0, double p1, int dtype, uint64_t seed,
       v = p0 * sqrt(-2.0 * log(unit_open(a))) * cos(6.283185307179586476925 * unit_open(b));
       if (kind == 3 && v < 0.0) v = 0.0;
     }
-    if (dtype == 3) ((uint32_t*)out)[n] = float_to_tf32_rne((float)v);
+    if (dtype == 5 || dtype == 6) ((uint8_t*)out)[n] = sp24_inputs_to_fp8(v, dtype == 6);
+    else if (dtype == 3) ((uint32_t*)out)[n] = float_to_tf32_rne((float)v);
     else if (dtype == 2) ((int8_t*)out)[n] = (int8_t)v;
     else if (dtype == 1) ((uint16_t*)out)[n] = float_to_bf16_rne((float)v);
     else ((uint16_t*)out)[n] = double_to_half_rne(v);

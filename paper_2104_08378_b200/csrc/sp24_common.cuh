@@ -12,14 +12,18 @@ __host__ __device__ inline int elem_bytes(sp24_dtype t) {
   switch (t) {
     case SP24_F16:
     case SP24_BF16: return 2;
-    case SP24_I8: return 1;
+    case SP24_I8:
+    case SP24_E4M3:
+    case SP24_E5M2: return 1;
     case SP24_F32:
     case SP24_I32: return 4;
   }
   return 0;
 }
 
-inline bool is_ab_type(sp24_dtype t) { return t == SP24_F16 || t == SP24_BF16 || t == SP24_I8; }
+inline bool is_fp8(sp24_dtype t) { return t == SP24_E4M3 || t == SP24_E5M2; }
+// types of the 2:4 pattern (SP24_F32, the 1:2 pattern, is handled apart)
+inline bool is_ab_type(sp24_dtype t) { return t == SP24_F16 || t == SP24_BF16 || t == SP24_I8 || is_fp8(t); }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -66,6 +66,9 @@ struct GemmParams {
   float out_inv_scale;
 };
 
+// MMA kinds: 0 = f16 / bf16, 1 = int8, 2 = tf32, 3 = 8-bit floating point (e4m3 / e5m2)
+__host__ __device__ constexpr bool one_byte_operands(int kind) { return kind == 1 || kind == 3; }
+
 template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK, bool B_MN>
 struct Cfg {
   // 128-byte atoms per stage: sparse A is half as wide as B; the dense variant with two
@@ -75,7 +78,7 @@ struct Cfg {
   static constexpr int kBRows = BLOCK_N / CTAS;                    // B rows (N) this CTA loads
   static constexpr int kABlockBytes = kABoxes * kBlockM * kAtomBytes;  // one m-block
   static constexpr int kABytes = MBLK * kABlockBytes;
-  static constexpr int kAtomElems = KIND == 0 ? 64 : (KIND == 1 ? 128 : 32);  // elements per 128-byte row
+  static constexpr int kAtomElems = KIND == 0 ? 64 : (one_byte_operands(KIND) ? 128 : 32);  // elements per 128-byte row
   static constexpr int kKPerStage = kAtomElems * kBBoxes;  // logical K per stage
   // B with N contiguous (MN-major operand): 128-byte chunks along N, each kKPerStage k-rows of 128 bytes
   static constexpr int kBChunkElems = kAtomElems;
@@ -83,7 +86,7 @@ struct Cfg {
   static constexpr int kBChunkBytes = kKPerStage * kAtomBytes;
   static constexpr int kBKStepBytes = (SPARSE ? 2 : 1) * (kAtomElems / 4) * kAtomBytes;  // k-rows of one MMA
   static constexpr int kBBytes = B_MN ? kBChunks * kBChunkBytes : kBBoxes * kBRows * kAtomBytes;
-  static constexpr int kEBlocks = SPARSE ? (KIND == 1 ? 2 : 1) : 0;  // 2048-byte metadata blocks per m-block and stage
+  static constexpr int kEBlocks = SPARSE ? (one_byte_operands(KIND) ? 2 : 1) : 0;  // 2048-byte metadata blocks per m-block and stage
   static constexpr int kEBlockBytes = kEBlocks * 2048;
   static constexpr int kEBytes = MBLK * kEBlockBytes;
   static constexpr int kEAlloc = (kEBytes + 1023) / 1024 * 1024;
@@ -147,7 +150,8 @@ __device__ __forceinline__ uint32_t make_idesc(bool sparse, bool b_mn_major, int
   uint32_t d = 0;
   d |= (sparse ? 1u : 0u) << 2;
   d |= (KIND == 1 ? 2u : 1u) << 4;                 // accumulator: int32 / fp32
-  uint32_t fmt = KIND == 0 ? (uint32_t)a_fmt : (KIND == 1 ? 1u : 2u);  // f16 = 0, bf16 = 1, tf32 = 2; int8: 1 = signed
+  // kind f16: f16 = 0, bf16 = 1; tf32: 2; int8: 1 = signed; 8-bit floats: e4m3 = 0, e5m2 = 1
+  uint32_t fmt = (KIND == 0 || KIND == 3) ? (uint32_t)a_fmt : (KIND == 1 ? 1u : 2u);
   d |= fmt << 7;
   d |= fmt << 10;
   d |= (b_mn_major ? 1u : 0u) << 16;               // A is always K-major
@@ -520,7 +524,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 uint64_t da = ptx::smem_desc(saj + k * 32, true, 1024);
                 uint64_t db = B_MN ? ptx::smem_desc(sb + k * C::kBKStepBytes, true, 1024, C::kBChunkBytes)
                                    : ptx::smem_desc(sb + (k >> 1) * C::kBRows * kAtomBytes + (k & 1) * 64, true, 1024);
-                if (KIND != 1) {
+                if (!one_byte_operands(KIND)) {
                   // one 32-bit metadata column per instruction: even-aligned address + selector
                   ptx::mma_sparse<KIND, CTAS>(d_tmem, da, db, e_tmem + (k & ~1), idesc | (uint32_t)(k & 1), accumulate);
                 } else {
@@ -777,7 +781,7 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
                    cudaStream_t stream) {
   using C = Cfg<KIND, SPARSE, BLOCK_N, CTAS, MBLK, B_MN>;
   GemmParams p = base;
-  const int es = KIND == 0 ? 2 : (KIND == 1 ? 1 : 4);
+  const int es = KIND == 0 ? 2 : (one_byte_operands(KIND) ? 1 : 4);
   const int tile_m = kBlockM * CTAS * MBLK;
   p.m_tiles = (int)((d->M + tile_m - 1) / tile_m);
   p.n_tiles = (int)((d->N + BLOCK_N - 1) / BLOCK_N);
@@ -867,16 +871,19 @@ static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, con
                                  bool& has_c, float& falpha, float& fbeta, bool dequant = false) {
   SP24_RETURN_IF(d == nullptr || (!dequant && (alpha == nullptr || beta == nullptr)), SP24_ERR_NULL);
   const bool tf32 = d->ab_type == SP24_F32;
-  const bool fp = d->ab_type == SP24_F16 || d->ab_type == SP24_BF16 || tf32;
+  const bool f8 = is_fp8(d->ab_type);
+  const bool fp = d->ab_type == SP24_F16 || d->ab_type == SP24_BF16 || tf32 || f8;
   SP24_RETURN_IF(!fp && d->ab_type != SP24_I8, SP24_ERR_DTYPE);
   SP24_RETURN_IF(tf32 && (d->cd_type != SP24_F32 || d->order_b != SP24_COL_MAJOR), SP24_ERR_UNSUPPORTED);
+  SP24_RETURN_IF(f8 && d->order_b != SP24_COL_MAJOR, SP24_ERR_UNSUPPORTED);
   if (dequant)
     SP24_RETURN_IF(fp || (d->cd_type != SP24_BF16 && d->cd_type != SP24_F16 && d->cd_type != SP24_F32 &&
                           d->cd_type != SP24_I8),
                    SP24_ERR_DTYPE);
+  else if (f8) SP24_RETURN_IF(d->cd_type != SP24_F16 && d->cd_type != SP24_BF16 && d->cd_type != SP24_F32, SP24_ERR_DTYPE);
   else if (fp) SP24_RETURN_IF(d->cd_type != d->ab_type && d->cd_type != SP24_F32, SP24_ERR_DTYPE);
   else SP24_RETURN_IF(d->cd_type != SP24_I32, SP24_ERR_DTYPE);
-  const int64_t mult = fp ? 16 : 32;
+  const int64_t mult = elem_bytes(d->ab_type) == 1 ? 32 : 16;
   SP24_RETURN_IF(d->M < 0 || d->N < 0 || d->K <= 0, SP24_ERR_SHAPE);
   SP24_RETURN_IF(d->M % mult || d->N % mult || d->K % mult, SP24_ERR_SHAPE);
   SP24_RETURN_IF(d->M > (int64_t(1) << 30) || d->N > (int64_t(1) << 30) || d->K > (int64_t(1) << 30), SP24_ERR_SHAPE);
@@ -957,12 +964,12 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   p.D = D;
   p.status = static_cast<uint32_t*>(workspace);
   p.alpha = falpha; p.beta = fbeta;
-  p.a_fmt = d->ab_type == SP24_BF16 ? 1 : 0;
+  p.a_fmt = (d->ab_type == SP24_BF16 || d->ab_type == SP24_E5M2) ? 1 : 0;
   p.cd_type = (int)d->cd_type;
   p.has_c = has_c ? 1 : 0;
   p.cd_col_major = d->order_d == SP24_COL_MAJOR ? 1 : 0;
   const bool sparse = !d->a_is_dense;
-  const bool i8 = d->ab_type == SP24_I8, tf32 = d->ab_type == SP24_F32;
+  const bool i8 = d->ab_type == SP24_I8, tf32 = d->ab_type == SP24_F32, f8 = is_fp8(d->ab_type);
   // Tile choice.  Large problems (at least six waves of tiles): a pair of CTAs with two m-blocks
   // each, 512 x 224 tiles: least operand traffic per flop.  Medium: a pair with one m-block, 256 x 224,
   // epilogue overlapped.  Small: single CTAs, 128 x 128.  (224: two fp32 accumulators plus the
@@ -985,11 +992,13 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
 #define SP24_LAUNCH(K_, BN, CT, MB, MN)                                                               \
   (sparse ? launch<K_, true, BN, CT, MB, MN>(d, p, A, meta, B, s) : launch<K_, false, BN, CT, MB, MN>(d, p, A, meta, B, s))
 #define SP24_DISPATCH(CT, BN, MB)                                                                     \
-  if (ctas == CT && block_n == BN && mblk == MB && !b_mn && !tf32) return i8 ? SP24_LAUNCH(1, BN, CT, MB, false) : SP24_LAUNCH(0, BN, CT, MB, false);
+  if (ctas == CT && block_n == BN && mblk == MB && !b_mn && !tf32 && !f8) return i8 ? SP24_LAUNCH(1, BN, CT, MB, false) : SP24_LAUNCH(0, BN, CT, MB, false);
 #define SP24_DISPATCH_TF32(CT, BN, MB)                                                                \
   if (ctas == CT && block_n == BN && mblk == MB && !b_mn && tf32) return SP24_LAUNCH(2, BN, CT, MB, false);
+#define SP24_DISPATCH_F8(CT, BN, MB)                                                                  \
+  if (ctas == CT && block_n == BN && mblk == MB && !b_mn && f8) return SP24_LAUNCH(3, BN, CT, MB, false);
 #define SP24_DISPATCH_MN(CT, BN, MB)                                                                  \
-  if (ctas == CT && block_n == BN && mblk == MB && b_mn) return i8 ? SP24_LAUNCH(1, BN, CT, MB, true) : SP24_LAUNCH(0, BN, CT, MB, true);
+  if (ctas == CT && block_n == BN && mblk == MB && b_mn && !tf32 && !f8) return i8 ? SP24_LAUNCH(1, BN, CT, MB, true) : SP24_LAUNCH(0, BN, CT, MB, true);
   SP24_DISPATCH(1, 128, 1)
   SP24_DISPATCH(2, 224, 1)
   SP24_DISPATCH(2, 224, 2)
@@ -998,12 +1007,16 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   SP24_DISPATCH_TF32(1, 128, 1)
   SP24_DISPATCH_TF32(2, 224, 1)
   SP24_DISPATCH_TF32(2, 224, 2)
+  SP24_DISPATCH_F8(1, 128, 1)
+  SP24_DISPATCH_F8(2, 224, 1)
+  SP24_DISPATCH_F8(2, 224, 2)
   SP24_DISPATCH_MN(1, 128, 1)
   SP24_DISPATCH_MN(2, 224, 1)
   SP24_DISPATCH_MN(2, 224, 2)
 #undef SP24_DISPATCH
 #undef SP24_DISPATCH_MN
 #undef SP24_DISPATCH_TF32
+#undef SP24_DISPATCH_F8
 #undef SP24_LAUNCH
   return SP24_ERR_UNSUPPORTED;
 }
@@ -1033,7 +1046,7 @@ extern "C" sp24_status sp24_conv3x3_nhwc(const sp24_gemm_desc* d, int64_t Nb, in
   SP24_RETURN_IF(d->N != Nb * H * W || d->K != 9 * Cin, SP24_ERR_SHAPE);
   SP24_RETURN_IF(!is_ab_type(d->ab_type), SP24_ERR_DTYPE);
   // a shared-memory stage holds 128 (16-bit) or 256 (int8) consecutive k = channels of ONE filter tap
-  const int64_t per_stage = d->ab_type == SP24_I8 ? 256 : 128;
+  const int64_t per_stage = elem_bytes(d->ab_type) == 1 ? 256 : 128;
   SP24_RETURN_IF(Cin % per_stage != 0, SP24_ERR_SHAPE);
   SP24_RETURN_IF(H > 32767 || W > 32767 || Nb > (int64_t(1) << 30), SP24_ERR_SHAPE);
   SP24_RETURN_IF(d->order_b != SP24_COL_MAJOR, SP24_ERR_UNSUPPORTED);

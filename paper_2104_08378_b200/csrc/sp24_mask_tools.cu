@@ -191,7 +191,7 @@ using namespace sp24;
 
 extern "C" sp24_status sp24_kept_magnitude(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx,
                                            const int32_t* perm, double* result, void* stream) {
-  SP24_RETURN_IF(!is_ab_type(t), SP24_ERR_DTYPE);
+  SP24_RETURN_IF(!is_ab_type(t) || is_fp8(t), SP24_ERR_DTYPE);
   SP24_RETURN_IF(M < 0 || K < 0 || K % 4 != 0, SP24_ERR_SHAPE);
   SP24_RETURN_IF(result == nullptr, SP24_ERR_NULL);
   if (M == 0 || K == 0) return SP24_OK;
@@ -236,7 +236,7 @@ extern "C" sp24_status sp24_apply_mask(sp24_dtype t, int64_t M, int64_t K, const
 
 extern "C" sp24_status sp24_prune_2d(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx, void* y, int64_t ldy,
                                      void* stream) {
-  SP24_RETURN_IF(!is_ab_type(t), SP24_ERR_DTYPE);
+  SP24_RETURN_IF(!is_ab_type(t) || is_fp8(t), SP24_ERR_DTYPE);
   SP24_RETURN_IF(M < 0 || K < 0 || K % 4 != 0 || M % 4 != 0, SP24_ERR_SHAPE);
   if (M == 0 || K == 0) return SP24_OK;
   SP24_RETURN_IF(x == nullptr || y == nullptr, SP24_ERR_NULL);

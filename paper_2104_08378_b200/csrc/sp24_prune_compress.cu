@@ -46,6 +46,11 @@ struct Group8 {
   }
 };
 
+// Magnitude keys of 8-bit elements: |x| for int8 (-128 -> 0x80 = 128, no saturation), the seven
+// bits below the sign for the 8-bit floating-point types (`f8` != 0).
+__device__ __forceinline__ uint32_t keys8(uint32_t w, int f8) { return f8 ? (w & 0x7F7F7F7Fu) : __vabs4(w); }
+__device__ __forceinline__ uint32_t key8(uint32_t e, int f8) { return f8 ? (e & 0x7Fu) : (uint32_t)abs((int)(int8_t)e); }
+
 __device__ __forceinline__ uint4 ld_stream(const void* p) { return __ldcs(reinterpret_cast<const uint4*>(p)); }
 __device__ __forceinline__ void st_stream(void* p, uint4 v) { __stcs(reinterpret_cast<uint4*>(p), v); }
 
@@ -53,7 +58,7 @@ __device__ __forceinline__ void st_stream(void* p, uint4 v) { __stcs(reinterpret
 // Any alignment / leading dimension: one thread per group, element-wise accesses.
 template <typename T>
 __global__ void prune_scalar_kernel(const T* __restrict__ x, int64_t ldx, T* y, int64_t ldy, int64_t groups_per_row,
-                                    int64_t total) {
+                                    int64_t total, int f8) {
   int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (id >= total) return;
   int64_t row = id / groups_per_row, g = id - row * groups_per_row;
@@ -63,7 +68,7 @@ __global__ void prune_scalar_kernel(const T* __restrict__ x, int64_t ldx, T* y, 
 #pragma unroll
   for (int p = 0; p < 4; ++p) {
     e[p] = src[p];
-    key[p] = sizeof(T) == 2 ? (uint32_t)((uint16_t)e[p] & 0x7FFFu) : (uint32_t)abs((int)(int8_t)e[p]);
+    key[p] = sizeof(T) == 2 ? (uint32_t)((uint16_t)e[p] & 0x7FFFu) : key8((uint32_t)(uint8_t)e[p], f8);
   }
   uint32_t m = keep_mask4(key[0], key[1], key[2], key[3]);
   T* dst = y + row * ldy + 4 * g;
@@ -149,7 +154,7 @@ __device__ __forceinline__ uint32_t prune_selectors(uint32_t idx) {
 }
 
 template <int ES>
-__device__ __forceinline__ uint4 prune_vec(uint4 v, const uint32_t* table) {
+__device__ __forceinline__ uint4 prune_vec(uint4 v, const uint32_t* table, int f8) {
   if (ES == 2) {
     const uint32_t s0 = table[selection_index(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu)];
     const uint32_t s1 = table[selection_index(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu)];
@@ -159,7 +164,7 @@ __device__ __forceinline__ uint4 prune_vec(uint4 v, const uint32_t* table) {
   uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
-    const uint32_t a = __vabs4(w[g]);  // -128 -> 0x80 = 128, no saturation
+    const uint32_t a = keys8(w[g], f8);
     w[g] = __byte_perm(w[g], 0, table[selection_index(__byte_perm(a, 0, 0x4140), __byte_perm(a, 0, 0x4342))]);
   }
   return make_uint4(w[0], w[1], w[2], w[3]);
@@ -169,7 +174,7 @@ __device__ __forceinline__ uint4 prune_vec(uint4 v, const uint32_t* table) {
 template <int ES, int UNROLL>
 __global__ void __launch_bounds__(kThreads) prune_vec_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
                                                              uint8_t* y, int64_t row_bytes_y, int64_t vpr,
-                                                             int64_t rows) {
+                                                             int64_t rows, int f8) {
   __shared__ uint32_t table[64];
   {
     const int t = threadIdx.y * blockDim.x + threadIdx.x;
@@ -190,7 +195,7 @@ __global__ void __launch_bounds__(kThreads) prune_vec_kernel(const uint8_t* __re
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
       const uint32_t c = c0 + u * blockDim.x;
-      if (c < vpr) st_stream(yr + c * 16u, prune_vec<ES>(v[u], table));
+      if (c < vpr) st_stream(yr + c * 16u, prune_vec<ES>(v[u], table, f8));
     }
   }
 }
@@ -278,7 +283,7 @@ __global__ void __launch_bounds__(kThreads, 4) compress8_kernel(const uint8_t* _
                                                              uint8_t* __restrict__ vals, int64_t row_bytes_v,
                                                              uint8_t* __restrict__ meta, int64_t M, int64_t K,
                                                              int64_t rows_pad, int64_t chunks_pad,
-                                                             unsigned long long* dropped) {
+                                                             unsigned long long* dropped, int f8) {
   __shared__ uint32_t table[64];
   build_selection_table(table);
   const uint32_t chunks = (uint32_t)(K >> 4), cpad = (uint32_t)chunks_pad, KB = (uint32_t)(chunks_pad >> 3);
@@ -313,12 +318,12 @@ __global__ void __launch_bounds__(kThreads, 4) compress8_kernel(const uint8_t* _
         mbits = 0;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-          const uint32_t a = __vabs4(w[g]);  // -128 -> 0x80 = 128, no saturation
+          const uint32_t a = keys8(w[g], f8);
           const uint32_t e = table[selection_index(__byte_perm(a, 0, 0x4140), __byte_perm(a, 0, 0x4342))];
           const uint32_t pair = __byte_perm(w[g], 0, ((e >> 8) & 0xFFu) | 0x4400u);
           out[g >> 1] |= pair << (16 * (g & 1));
           mbits |= (e & 0xFu) << (4 * g);
-          if (COUNT) lost += __popc(Group8::nonzero(w[g]) & ~(e >> 4) & 0xFu);
+          if (COUNT) lost += __popc(Group8::nonzero(a) & ~(e >> 4) & 0xFu);
         }
         __stcs(reinterpret_cast<uint2*>(vr + chunk * 8u), make_uint2(out[0], out[1]));
       }
@@ -332,7 +337,7 @@ __global__ void __launch_bounds__(kThreads, 4) compress8_kernel(const uint8_t* _
 template <typename T>
 __global__ void compress_scalar_kernel(const T* __restrict__ x, int64_t ldx, T* __restrict__ vals, int64_t ldv,
                                        uint8_t* __restrict__ meta, int layout, int64_t M, int64_t K,
-                                       int64_t rows_pad, int64_t bytes_pad, unsigned long long* dropped) {
+                                       int64_t rows_pad, int64_t bytes_pad, unsigned long long* dropped, int f8) {
   constexpr int ES = sizeof(T);
   const int64_t total = rows_pad * bytes_pad, KB = bytes_pad >> 4;
   int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -348,7 +353,7 @@ __global__ void compress_scalar_kernel(const T* __restrict__ x, int64_t ldx, T* 
 #pragma unroll
       for (int p = 0; p < 4; ++p) {
         e[p] = src[p];
-        key[p] = ES == 2 ? (uint32_t)((uint16_t)e[p] & 0x7FFFu) : (uint32_t)abs((int)(int8_t)e[p]);
+        key[p] = ES == 2 ? (uint32_t)((uint16_t)e[p] & 0x7FFFu) : key8((uint32_t)(uint8_t)e[p], f8);
       }
       uint32_t m = keep_mask4(key[0], key[1], key[2], key[3]);
       uint32_t nib = mask_to_nibble(m);
@@ -601,7 +606,7 @@ extern "C" sp24_status sp24_prune(sp24_dtype t, int64_t M, int64_t K, const void
   SP24_RETURN_IF(ldx < K || ldy < K, SP24_ERR_STRIDE);
   if ((st = check_arch()) != SP24_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const int es = elem_bytes(t);
+  const int es = elem_bytes(t), f8 = is_fp8(t) ? 1 : 0;
   const bool vec = aligned16(x) && aligned16(y) && (ldx * es) % 16 == 0 && (ldy * es) % 16 == 0 && (K * es) % 16 == 0;
   if (vec) {
     constexpr int UNROLL = 4;
@@ -614,16 +619,16 @@ extern "C" sp24_status sp24_prune(sp24_dtype t, int64_t M, int64_t K, const void
     RowLaunch L(vpr, rows, UNROLL);
     int64_t rbx = ldx == K && ldy == K ? vpr * 16 : ldx * es, rby = ldx == K && ldy == K ? vpr * 16 : ldy * es;
     if (es == 2)
-      prune_vec_kernel<2, UNROLL><<<L.grid, L.block, 0, s>>>((const uint8_t*)x, rbx, (uint8_t*)y, rby, vpr, rows);
+      prune_vec_kernel<2, UNROLL><<<L.grid, L.block, 0, s>>>((const uint8_t*)x, rbx, (uint8_t*)y, rby, vpr, rows, f8);
     else
-      prune_vec_kernel<1, UNROLL><<<L.grid, L.block, 0, s>>>((const uint8_t*)x, rbx, (uint8_t*)y, rby, vpr, rows);
+      prune_vec_kernel<1, UNROLL><<<L.grid, L.block, 0, s>>>((const uint8_t*)x, rbx, (uint8_t*)y, rby, vpr, rows, f8);
   } else {
     int64_t gpr = K / 4, total = M * gpr;
     unsigned blocks = blocks_for(total, kThreads);
     if (es == 2)
-      prune_scalar_kernel<uint16_t><<<blocks, kThreads, 0, s>>>((const uint16_t*)x, ldx, (uint16_t*)y, ldy, gpr, total);
+      prune_scalar_kernel<uint16_t><<<blocks, kThreads, 0, s>>>((const uint16_t*)x, ldx, (uint16_t*)y, ldy, gpr, total, 0);
     else
-      prune_scalar_kernel<int8_t><<<blocks, kThreads, 0, s>>>((const int8_t*)x, ldx, (int8_t*)y, ldy, gpr, total);
+      prune_scalar_kernel<int8_t><<<blocks, kThreads, 0, s>>>((const int8_t*)x, ldx, (int8_t*)y, ldy, gpr, total, f8);
   }
   return cuda_status(cudaGetLastError());
 }
@@ -660,7 +665,7 @@ extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const v
   SP24_RETURN_IF(ldx < K || ldv < K / 2, SP24_ERR_STRIDE);
   if ((st = check_arch()) != SP24_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const int es = elem_bytes(t);
+  const int es = elem_bytes(t), f8 = is_fp8(t) ? 1 : 0;
   const bool hw = l == SP24_META_TCGEN05;
   const int64_t rows_pad = hw ? (M + 127) / 128 * 128 : M;
   const int64_t k_pad = hw ? (K + 255) / 256 * 256 : K;
@@ -696,7 +701,7 @@ extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const v
       const int variant = (dropped ? 4 : 0) | (hw ? 2 : 0) | (full ? 1 : 0);
 #define SP24_C8(COUNT, HW, FULL)                                                                          \
   compress8_kernel<UNROLL, COUNT, HW, FULL><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, M, K, \
-                                                                       rows_pad, chunks_pad, dropped)
+                                                                       rows_pad, chunks_pad, dropped, f8)
       switch (variant) {
         case 0: SP24_C8(false, false, false); break;
         case 1: SP24_C8(false, false, true); break;
@@ -715,11 +720,11 @@ extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const v
     if (es == 2)
       compress_scalar_kernel<uint16_t><<<blocks, kThreads, 0, s>>>((const uint16_t*)x, ldx, (uint16_t*)vals, ldv,
                                                                    (uint8_t*)meta, (int)l, M, K, rows_pad, bytes_pad,
-                                                                   dropped);
+                                                                   dropped, 0);
     else
       compress_scalar_kernel<int8_t><<<blocks, kThreads, 0, s>>>((const int8_t*)x, ldx, (int8_t*)vals, ldv,
                                                                  (uint8_t*)meta, (int)l, M, K, rows_pad, bytes_pad,
-                                                                 dropped);
+                                                                 dropped, f8);
   }
   return cuda_status(cudaGetLastError());
 }

@@ -199,64 +199,49 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t smem_addr, bool swizzle12
 
 // ---- MMA -------------------------------------------------------------------------------------------
 // KIND 0: kind::f16 (fp16 / bf16 operands, fp32 accumulate); KIND 1: kind::i8 (int32 accumulate);
-// KIND 2: kind::tf32 (fp32 storage, tf32 multiply, fp32 accumulate).
+// KIND 2: kind::tf32 (fp32 storage, tf32 multiply, fp32 accumulate); KIND 3: kind::f8f6f4 with 8-bit
+// floating-point operands (e4m3 / e5m2, fp32 accumulate).
+#define SP24_MMA_DENSE(GROUP, KINDNAME)                                                                       \
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"                                             \
+               "tcgen05.mma.cta_group::" GROUP ".kind::" KINDNAME " [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem), \
+               "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)                                         \
+               : "memory")
+#define SP24_MMA_SPARSE(GROUP, KINDNAME)                                                                      \
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"                                             \
+               "tcgen05.mma.sp.cta_group::" GROUP ".kind::" KINDNAME " [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"( \
+                   d_tmem),                                                                                  \
+               "l"(a_desc), "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate)                            \
+               : "memory")
+
 template <int KIND, int CTAS>
 __device__ __forceinline__ void mma_dense(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate) {
-  if (KIND == 0 && CTAS == 1)
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc),
-                 "r"(idesc), "r"(accumulate) : "memory");
-  else if (KIND == 0 && CTAS == 2)
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc),
-                 "r"(idesc), "r"(accumulate) : "memory");
-  else if (KIND == 1 && CTAS == 1)
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc),
-                 "r"(idesc), "r"(accumulate) : "memory");
-  else if (KIND == 2 && CTAS == 1)
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc),
-                 "r"(idesc), "r"(accumulate) : "memory");
-  else if (KIND == 2 && CTAS == 2)
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc),
-                 "r"(idesc), "r"(accumulate) : "memory");
-  else
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc),
-                 "r"(idesc), "r"(accumulate) : "memory");
+  static_assert(KIND >= 0 && KIND <= 3 && (CTAS == 1 || CTAS == 2), "unknown MMA kind");
+  if (KIND == 0 && CTAS == 1) SP24_MMA_DENSE("1", "f16");
+  else if (KIND == 0) SP24_MMA_DENSE("2", "f16");
+  else if (KIND == 1 && CTAS == 1) SP24_MMA_DENSE("1", "i8");
+  else if (KIND == 1) SP24_MMA_DENSE("2", "i8");
+  else if (KIND == 2 && CTAS == 1) SP24_MMA_DENSE("1", "tf32");
+  else if (KIND == 2) SP24_MMA_DENSE("2", "tf32");
+  else if (CTAS == 1) SP24_MMA_DENSE("1", "f8f6f4");
+  else SP24_MMA_DENSE("2", "f8f6f4");
 }
 
 template <int KIND, int CTAS>
 __device__ __forceinline__ void mma_sparse(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t e_tmem,
                                            uint32_t idesc, uint32_t accumulate) {
-  if (KIND == 0 && CTAS == 1)
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                 "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"(d_tmem), "l"(a_desc),
-                 "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
-  else if (KIND == 0 && CTAS == 2)
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                 "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"(d_tmem), "l"(a_desc),
-                 "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
-  else if (KIND == 1 && CTAS == 1)
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                 "tcgen05.mma.sp.cta_group::1.kind::i8 [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"(d_tmem), "l"(a_desc),
-                 "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
-  else if (KIND == 2 && CTAS == 1)
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                 "tcgen05.mma.sp.cta_group::1.kind::tf32 [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"(d_tmem), "l"(a_desc),
-                 "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
-  else if (KIND == 2 && CTAS == 2)
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                 "tcgen05.mma.sp.cta_group::2.kind::tf32 [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"(d_tmem), "l"(a_desc),
-                 "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
-  else
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                 "tcgen05.mma.sp.cta_group::2.kind::i8 [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"(d_tmem), "l"(a_desc),
-                 "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
+  static_assert(KIND >= 0 && KIND <= 3 && (CTAS == 1 || CTAS == 2), "unknown MMA kind");
+  if (KIND == 0 && CTAS == 1) SP24_MMA_SPARSE("1", "f16");
+  else if (KIND == 0) SP24_MMA_SPARSE("2", "f16");
+  else if (KIND == 1 && CTAS == 1) SP24_MMA_SPARSE("1", "i8");
+  else if (KIND == 1) SP24_MMA_SPARSE("2", "i8");
+  else if (KIND == 2 && CTAS == 1) SP24_MMA_SPARSE("1", "tf32");
+  else if (KIND == 2) SP24_MMA_SPARSE("2", "tf32");
+  else if (CTAS == 1) SP24_MMA_SPARSE("1", "f8f6f4");
+  else SP24_MMA_SPARSE("2", "f8f6f4");
 }
+#undef SP24_MMA_DENSE
+#undef SP24_MMA_SPARSE
 
 // 128 lanes x 128 bits, shared memory -> tensor memory (metadata).
 template <int CTAS>

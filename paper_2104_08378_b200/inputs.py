@@ -29,7 +29,8 @@ TENSOR_A, TENSOR_B, TENSOR_C, TENSOR_TILES = 0, 1, 2, 3
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "csrc", "inputs_gen.c")
 _LIB = os.path.join(_HERE, "libsp24_inputs.so")
-_DTYPE = {"f16": 0, "bf16": 1, "i8": 2, "tf32": 3}
+_NP_STORAGE = {"i8": np.int8, "tf32": np.uint32, "e4m3": np.uint8, "e5m2": np.uint8}  # else uint16 bit patterns
+_DTYPE = {"f16": 0, "bf16": 1, "i8": 2, "tf32": 3, "e4m3": 5, "e5m2": 6}
 _lib = None
 
 
@@ -52,6 +53,8 @@ def _load():
         lib.sp24_inputs_fill.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_double,
                                          ctypes.c_int, u64, u64, u64, u64, ctypes.c_void_p]
         lib.sp24_inputs_fill.restype = None
+        lib.sp24_inputs_to_fp8.argtypes = [ctypes.c_double, ctypes.c_int]
+        lib.sp24_inputs_to_fp8.restype = ctypes.c_uint8
         _lib = lib
     return _lib
 
@@ -75,6 +78,11 @@ def to_storage(x: np.ndarray, dtype: str) -> np.ndarray:
         bits = np.ascontiguousarray(x.astype(np.float32)).view(np.uint32)
         rounding = ((bits >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
         return ((bits + rounding) >> np.uint32(16)).astype(np.uint16)
+    if dtype in ("e4m3", "e5m2"):
+        lib = _load()
+        flat = np.asarray(x, dtype=np.float64).ravel()
+        out = np.array([lib.sp24_inputs_to_fp8(float(v), 1 if dtype == "e5m2" else 0) for v in flat], dtype=np.uint8)
+        return out.reshape(np.shape(x))
     raise ValueError(dtype)
 
 
@@ -138,7 +146,7 @@ _KIND = {"normal": 0, "uniform": 1, "int8": 2, "relu_normal": 3}
 def _matrix(dist, dtype, seed, tensor_id, ncols, row0, row1) -> np.ndarray:
     """Rows row0..row1-1 of a (?, ncols) matrix whose element (r, c) has linear index r*ncols+c."""
     nrows = row1 - row0
-    out = np.empty((nrows, ncols), dtype=np.int8 if dtype == "i8" else (np.uint32 if dtype == "tf32" else np.uint16))
+    out = np.empty((nrows, ncols), dtype=_NP_STORAGE.get(dtype, np.uint16))
     if nrows == 0 or ncols == 0:
         return out
     p0 = float(dist[1]) if len(dist) > 1 else 0.0

@@ -258,6 +258,9 @@ def run_ours(args, cfg):
         torch.cuda.synchronize()
         ts = []
         for _ in range(reps):
+            # keep the GPU busy while the host enqueues, so that the host's launch latency is not
+            # part of the interval between the two events
+            torch.cuda._sleep(400000)
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
             fn()

@@ -277,7 +277,11 @@ sp24_status sp24_prune_2d(sp24_dtype t, int64_t M, int64_t K, const void* x, int
  * (M x N packed) to the device buffers the caller provides, runs sp24_compress (TCGEN05
  * layout) and sp24_gemm, and copies D (M x N packed) back.  All h_* are host pointers, all
  * d_* device pointers sized for the packed matrices (d_vals, d_meta as the size helpers
- * say).  Work is enqueued on `stream`; the caller synchronises. */
+ * say).  Work is enqueued on `stream`; the caller synchronises.  For M >= 16384 the work runs
+ * in up to eight row bands: each band's D is copied out on a second, library-owned stream
+ * (created once per device; `stream` is made to wait for it before the call returns) while
+ * the next band's A and C are copied in, so both directions of the host link are busy.  The status
+ * word in `workspace` then reflects the last band only. */
 sp24_status sp24_pipeline_host(const sp24_gemm_desc* d, const void* alpha, const void* h_A,
                                const void* h_B, const void* beta, const void* h_C, void* h_D,
                                void* d_A, void* d_vals, void* d_meta, void* d_B, void* d_C,

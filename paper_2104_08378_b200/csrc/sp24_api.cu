@@ -1,4 +1,6 @@
 // Size helpers, status strings, the architecture check and the host-buffer pipeline.
+#include <mutex>
+
 #include "sp24_common.cuh"
 
 namespace sp24 {
@@ -56,6 +58,37 @@ extern "C" size_t sp24_meta_bytes(sp24_dtype t, int64_t M, int64_t K, sp24_meta_
   return 0;
 }
 
+namespace {
+
+// Second stream and events of the host-buffer pipeline, created once per device and kept.
+constexpr int kMaxBands = 8;
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t band_done[kMaxBands] = {};
+  cudaEvent_t joined = nullptr;
+  bool ready = false;
+};
+
+sp24_status side_stream(SideStream** out) {
+  static std::mutex mu;
+  static SideStream per_device[64];
+  int dev = 0;
+  SP24_CUDA_CHECK(cudaGetDevice(&dev));
+  SP24_RETURN_IF(dev < 0 || dev >= 64, SP24_ERR_UNSUPPORTED);
+  std::lock_guard<std::mutex> lock(mu);
+  SideStream& ss = per_device[dev];
+  if (!ss.ready) {
+    SP24_CUDA_CHECK(cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking));
+    for (int b = 0; b < kMaxBands; ++b) SP24_CUDA_CHECK(cudaEventCreateWithFlags(&ss.band_done[b], cudaEventDisableTiming));
+    SP24_CUDA_CHECK(cudaEventCreateWithFlags(&ss.joined, cudaEventDisableTiming));
+    ss.ready = true;
+  }
+  *out = &ss;
+  return SP24_OK;
+}
+
+}  // namespace
+
 extern "C" sp24_status sp24_pipeline_host(const sp24_gemm_desc* d, const void* alpha, const void* h_A, const void* h_B,
                                           const void* beta, const void* h_C, void* h_D, void* d_A, void* d_vals,
                                           void* d_meta, void* d_B, void* d_C, void* d_D, void* workspace,
@@ -63,6 +96,7 @@ extern "C" sp24_status sp24_pipeline_host(const sp24_gemm_desc* d, const void* a
   SP24_RETURN_IF(d == nullptr || alpha == nullptr || beta == nullptr, SP24_ERR_NULL);
   SP24_RETURN_IF(!is_ab_type(d->ab_type), SP24_ERR_DTYPE);
   SP24_RETURN_IF(d->a_is_dense, SP24_ERR_UNSUPPORTED);
+  SP24_RETURN_IF(d->M < 0 || d->N < 0 || d->K <= 0, SP24_ERR_SHAPE);
   SP24_RETURN_IF(h_A == nullptr || h_B == nullptr || h_D == nullptr || d_A == nullptr || d_vals == nullptr ||
                      d_meta == nullptr || d_B == nullptr || d_D == nullptr,
                  SP24_ERR_NULL);
@@ -71,20 +105,58 @@ extern "C" sp24_status sp24_pipeline_host(const sp24_gemm_desc* d, const void* a
   SP24_RETURN_IF(has_c && (h_C == nullptr || d_C == nullptr), SP24_ERR_NULL);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t es = elem_bytes(d->ab_type), cs = elem_bytes(d->cd_type);
-  SP24_CUDA_CHECK(cudaMemcpyAsync(d_A, h_A, (size_t)d->M * d->K * es, cudaMemcpyHostToDevice, s));
+  SP24_RETURN_IF(cs == 0, SP24_ERR_DTYPE);
   SP24_CUDA_CHECK(cudaMemcpyAsync(d_B, h_B, (size_t)d->N * d->K * es, cudaMemcpyHostToDevice, s));
-  if (has_c) SP24_CUDA_CHECK(cudaMemcpyAsync(d_C, h_C, (size_t)d->M * d->N * cs, cudaMemcpyHostToDevice, s));
-  sp24_status st = sp24_compress(d->ab_type, d->M, d->K, d_A, d->K, d_vals, d->K / 2, d_meta, SP24_META_TCGEN05,
-                                 nullptr, stream);
-  if (st != SP24_OK) return st;
-  sp24_gemm_desc packed = *d;
-  packed.lda = d->K / 2;
-  packed.ldb = d->K;
-  packed.ldc = d->N;
-  packed.ldd = d->N;
-  st = sp24_gemm(&packed, alpha, d_vals, d_meta, d_B, beta, has_c ? d_C : nullptr, d_D, workspace, workspace_bytes,
-                 stream);
-  if (st != SP24_OK) return st;
-  SP24_CUDA_CHECK(cudaMemcpyAsync(h_D, d_D, (size_t)d->M * d->N * cs, cudaMemcpyDeviceToHost, s));
-  return SP24_OK;
+  sp24_status st = SP24_OK;
+  // Row bands of A / C / D (multiples of the 512-row tile): the copy-out of one band runs on a
+  // second stream while the caller's stream copies in the next band's A and C, compresses and
+  // multiplies it, so the two directions of the host link work at the same time.
+  int bands = (int)(d->M / 8192);
+  bands = bands < 1 ? 1 : (bands > kMaxBands ? kMaxBands : bands);
+  const int64_t band_rows = bands == 1 ? d->M : ((d->M + bands - 1) / bands + 511) / 512 * 512;
+  SideStream* ss = nullptr;
+  if (bands > 1 && (st = side_stream(&ss)) != SP24_OK) return st;
+  const size_t meta_block_bytes = sp24_meta_bytes(d->ab_type, 128, d->K, SP24_META_TCGEN05);  // per 128 rows
+  int issued = 0;
+  for (int b = 0; b < bands; ++b) {
+    const int64_t r0 = (int64_t)b * band_rows, r1 = r0 + band_rows < d->M ? r0 + band_rows : d->M;
+    if (r0 >= r1) break;
+    const size_t c_off = (size_t)r0 * d->N * cs, c_bytes = (size_t)(r1 - r0) * d->N * cs;
+    const size_t a_off = (size_t)r0 * d->K * es, v_off = (size_t)r0 * (d->K / 2) * es;
+    const size_t m_off = (size_t)(r0 / 128) * meta_block_bytes;
+    SP24_CUDA_CHECK(cudaMemcpyAsync(static_cast<char*>(d_A) + a_off, static_cast<const char*>(h_A) + a_off,
+                                    (size_t)(r1 - r0) * d->K * es, cudaMemcpyHostToDevice, s));
+    st = sp24_compress(d->ab_type, r1 - r0, d->K, static_cast<const char*>(d_A) + a_off, d->K,
+                       static_cast<char*>(d_vals) + v_off, d->K / 2, static_cast<char*>(d_meta) + m_off,
+                       SP24_META_TCGEN05, nullptr, stream);
+    if (st != SP24_OK) break;
+    if (has_c)
+      SP24_CUDA_CHECK(cudaMemcpyAsync(static_cast<char*>(d_C) + c_off, static_cast<const char*>(h_C) + c_off, c_bytes,
+                                      cudaMemcpyHostToDevice, s));
+    sp24_gemm_desc packed = *d;
+    packed.M = r1 - r0;
+    packed.lda = d->K / 2;
+    packed.ldb = d->K;
+    packed.ldc = d->N;
+    packed.ldd = d->N;
+    st = sp24_gemm(&packed, alpha, static_cast<const char*>(d_vals) + v_off,
+                   static_cast<const char*>(d_meta) + m_off, d_B, beta,
+                   has_c ? static_cast<const char*>(d_C) + c_off : nullptr, static_cast<char*>(d_D) + c_off, workspace,
+                   workspace_bytes, stream);
+    if (st != SP24_OK) break;
+    cudaStream_t out = s;
+    if (bands > 1) {
+      SP24_CUDA_CHECK(cudaEventRecord(ss->band_done[b], s));
+      SP24_CUDA_CHECK(cudaStreamWaitEvent(ss->stream, ss->band_done[b], 0));
+      out = ss->stream;
+      ++issued;
+    }
+    SP24_CUDA_CHECK(cudaMemcpyAsync(static_cast<char*>(h_D) + c_off, static_cast<const char*>(d_D) + c_off, c_bytes,
+                                    cudaMemcpyDeviceToHost, out));
+  }
+  if (issued) {  // the caller's stream ends behind every copy made on the second one
+    SP24_CUDA_CHECK(cudaEventRecord(ss->joined, ss->stream));
+    SP24_CUDA_CHECK(cudaStreamWaitEvent(s, ss->joined, 0));
+  }
+  return st;
 }

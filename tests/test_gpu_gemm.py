@@ -259,10 +259,13 @@ def test_implicit_conv3x3_matches_im2col_gemm(sp, case, dense):
                 check_fp(got, want, oracle.gemm_abs(vals_ref, meta_ref, Bt, ab, rows=rows, cols=(c0, c1)))
 
 
-def test_pipeline_host_entry_point(sp):
-    """sp24_pipeline_host: host buffers in, compress + GEMM on the device, D back in a host buffer."""
+@pytest.mark.parametrize("dims", [(384, 448, 512), (20000, 288, 128)])
+def test_pipeline_host_entry_point(sp, dims):
+    """sp24_pipeline_host: host buffers in, compress + GEMM on the device, D back in a host buffer.
+    The second case is large enough for the row-band pipeline (two bands, the last one ragged); it
+    runs twice in a row so that the second call's copies follow the first call's on both streams."""
     import ctypes
-    cfg = inputs.scaled(inputs.CONFIGS["gpt3_ffn_bf16"], M=384, N=448, K=512)
+    cfg = inputs.scaled(inputs.CONFIGS["gpt3_ffn_bf16"], M=dims[0], N=dims[1], K=dims[2])
     M, N, K = cfg.M, cfg.N, cfg.K
     A, Bt, Cm = inputs.gen_A(cfg), inputs.gen_Bt(cfg), inputs.gen_C(cfg)
     hA, hB, hC = (torch.from_numpy(a.view(np.int16)).pin_memory() for a in (A, Bt, Cm))
@@ -277,11 +280,13 @@ def test_pipeline_host_entry_point(sp):
     desc = sp.make_desc("bf16", "bf16", M, N, K, K // 2, K, N, N)
     al, be = ctypes.c_float(1.0), ctypes.c_float(1.0)
     vp = lambda t: ctypes.c_void_p(t.data_ptr())  # noqa: E731
-    st = sp.lib.sp24_pipeline_host(ctypes.byref(desc), ctypes.byref(al), vp(hA), vp(hB), ctypes.byref(be), vp(hC), vp(hD),
-                                   vp(dA), vp(dV), vp(dM), vp(dB), vp(dC), vp(dD), vp(ws), 256,
-                                   torch.cuda.current_stream().cuda_stream)
-    assert st == 0
+    for _ in range(2):
+        st = sp.lib.sp24_pipeline_host(ctypes.byref(desc), ctypes.byref(al), vp(hA), vp(hB), ctypes.byref(be), vp(hC),
+                                       vp(hD), vp(dA), vp(dV), vp(dM), vp(dB), vp(dC), vp(dD), vp(ws), 256,
+                                       torch.cuda.current_stream().cuda_stream)
+        assert st == 0
     torch.cuda.synchronize()
+    assert sp.gemm_status(ws) == 0
     vals_ref, meta_ref, _ = oracle.compress(A, "bf16")
     ref = oracle.gemm_sparse(vals_ref, meta_ref, Bt, "bf16", 1.0, 1.0, Cm, "bf16")
     got = oracle.bits_to_float64(hD.numpy().view(np.uint16), "bf16")

@@ -54,6 +54,7 @@ struct GemmParams {
   int32_t a_fmt;      // 0 f16, 1 bf16 (kind::f16); ignored for int8
   int32_t cd_type;    // sp24_dtype of C / D
   int32_t has_c;
+  int32_t stages, epi_bytes;  // shared memory: ring stages and bytes of epilogue staging
   int32_t band;       // m-tiles per band of the tile sweep
   int32_t cd_col_major;  // C and D stored M-contiguous (the [tokens, out_features] layout)
   // implicit 3x3 convolution: B is the im2col view of an NHWC activation (never materialised)
@@ -92,15 +93,16 @@ struct Cfg {
   static constexpr int kEAlloc = (kEBytes + 1023) / 1024 * 1024;
   static constexpr int kStageBytes = kABytes + kBBytes + kEAlloc;
   // shared memory: [stage ring | epilogue staging | barriers]; 1 KB of slack for the 1024-byte alignment
+  // The split between ring stages and epilogue staging is made per launch (the output type
+  // decides how much staging is useful).
   static constexpr int kSmemLimit = 232448 - 1024 - 512;
-  static constexpr int kStagesFit = (kSmemLimit - 16384) / kStageBytes;
-  static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
-  static constexpr int kEpiBytes = (kSmemLimit - kStages * kStageBytes >= 32768) ? 32768 : 16384;  // all 4 warps
+  static constexpr int kMaxStages = 8;
+  static constexpr int kMinStagesFit = (kSmemLimit - 16384) / kStageBytes;  // with the smallest staging
   static constexpr int kAccStages = MBLK == 2 ? 1 : ((2 * BLOCK_N + (SPARSE ? 32 : 0) <= (int)kTmemCols) ? 2 : 1);
   static constexpr int kECol = kAccStages * MBLK * BLOCK_N;        // first metadata column in tensor memory
   static constexpr int kMmasPerStage = SPARSE ? 4 : 4 * kBBoxes;   // per m-block
-  static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
-  static_assert(kStages >= 2, "need at least two stages");
+  static constexpr int kSmemBytes = 232448;  // always the whole opt-in maximum
+  static_assert(kMinStagesFit >= 2, "need at least two stages");
   static_assert(BLOCK_N % 32 == 0, "the epilogue moves 32-column boxes");
   static_assert(kStageBytes % 1024 == 0, "stages must keep the 1024-byte alignment of the atoms");
   static_assert(kECol + (SPARSE ? 2 * MBLK * 8 : 0) <= (int)kTmemCols, "tensor memory overflow");
@@ -353,8 +355,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   extern __shared__ uint8_t smem_raw[];
   // Operand atoms need 1024-byte alignment for the 128-byte swizzle.
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* epi = smem + C::kStages * C::kStageBytes;
-  Shared* sh = reinterpret_cast<Shared*>(epi + C::kEpiBytes);
+  uint8_t* epi = smem + p.stages * C::kStageBytes;
+  Shared* sh = reinterpret_cast<Shared*>(epi + p.epi_bytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t cta_rank = CTAS == 2 ? ptx::cluster_ctarank() : 0;
@@ -362,7 +364,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   const int num_tiles = p.m_tiles * p.n_tiles;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < C::kStages; ++s) {
+    for (int s = 0; s < p.stages; ++s) {
       ptx::mbar_init(&sh->full[s], 1);
       ptx::mbar_init(&sh->empty[s], 1);
     }
@@ -471,7 +473,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               else ptx::tma_load_2d_pair(sb + i * C::kBRows * kAtomBytes, &map_b, full, 0, x, col0);
             }
           }
-          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
       }
     }
@@ -541,7 +543,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           // the stage may be refilled once these MMAs have read it
           if (CTAS == 1) ptx::tc_commit(&sh->empty[stage]);
           else ptx::tc_commit_pair(&sh->empty[stage], 3);
-          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         if (CTAS == 1) ptx::tc_commit(&sh->tmem_full[acc]);
@@ -560,10 +562,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int buf_bytes = 1024 * cs;
     // Both warps of a quarter work (alternate boxes) when each can have a staging buffer of its own;
     // otherwise the second one only takes part in handing the accumulators back.
-    const int split = (C::kEpiBytes / kEpiWarps >= buf_bytes) ? 2 : 1;
+    const int split = (p.epi_bytes / kEpiWarps >= buf_bytes) ? 2 : 1;
     const int first_it = ew >> 2;
     const bool active = first_it < split;
-    const int warp_bytes = C::kEpiBytes / (4 * split);
+    const int warp_bytes = p.epi_bytes / (4 * split);
     const int nbuf = min(4, warp_bytes / buf_bytes);  // staging buffers of this warp: 1, 2 or 4
     const int ahead = nbuf > 1 ? nbuf - 1 : 1;      // boxes the C loads run ahead (their latency is what the epilogue waits on)
     // stores that may still be reading their buffer when the next buffer is claimed: with C the
@@ -823,6 +825,16 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
     if (st != SP24_OK) return st;
   } else {
     map_c = map_d;
+  }
+  // Shared-memory split.  The ring comes first (these kernels are bound by the operand feed: one
+  // stage less cost the int8 configuration 9 %); staging gets what is left, up to two boxes per
+  // epilogue warp (16 boxes of 1024 output elements), in powers of two from 16 KB.
+  {
+    p.stages = C::kMinStagesFit > C::kMaxStages ? C::kMaxStages : C::kMinStagesFit;
+    const int room = C::kSmemLimit - p.stages * C::kStageBytes;
+    int epi = 16384;
+    while (epi < 16 * 1024 * cs && 2 * epi <= room) epi *= 2;
+    p.epi_bytes = epi;
   }
   auto kernel = gemm_kernel<KIND, SPARSE, BLOCK_N, CTAS, MBLK, B_MN>;
   {

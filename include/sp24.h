@@ -125,6 +125,17 @@ sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const void* x, int
                           void* vals, int64_t ldv, void* meta, sp24_meta_layout l,
                           unsigned long long* dropped_nonzeros, void* stream);
 
+/* sp24_prune and sp24_compress in ONE pass over x (Section 4.1 step 2 followed by the storage
+ * format of Section 3.1): y receives what sp24_prune(x) would write, vals / meta / dropped what
+ * sp24_compress(x) would, bit for bit; x is read once instead of twice and the pruned matrix is
+ * not re-read.  Arguments as for the two calls; y may be the same buffer as x.  Operands the
+ * vectorised kernels cannot take (see sp24_prune) and the SP24_F32 1:2 pattern run as the two
+ * separate passes. */
+sp24_status sp24_prune_compress(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx,
+                                void* y, int64_t ldy, void* vals, int64_t ldv, void* meta,
+                                sp24_meta_layout l, unsigned long long* dropped_nonzeros,
+                                void* stream);
+
 /* Inverse of sp24_compress (the metadata is what decodes the format, Section 3.1):
  * y is M x K row-major (ldy >= K) with y[i, 4g+p_t] = vals[i, 2g+t] and +0 elsewhere. */
 sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals, int64_t ldv,

@@ -29,7 +29,7 @@ _FROM_TORCH = {torch.float16: "f16", torch.bfloat16: "bf16", torch.int8: "i8", t
 
 EXPORTS = [
     "sp24_status_string", "sp24_values_bytes", "sp24_meta_bytes", "sp24_prune", "sp24_compress",
-    "sp24_decompress", "sp24_gemm_workspace_bytes", "sp24_gemm", "sp24_gemm_status",
+    "sp24_decompress", "sp24_prune_compress", "sp24_gemm_workspace_bytes", "sp24_gemm", "sp24_gemm_status",
     "sp24_im2col_nhwc_3x3", "sp24_pipeline_host", "sp24_gemm_static_ws", "sp24_gemm_i8_dequant",
     "sp24_conv3x3_nhwc", "sp24_kept_magnitude", "sp24_apply_mask", "sp24_prune_2d",
 ]
@@ -65,6 +65,7 @@ def _load() -> ctypes.CDLL:
     lib.sp24_prune.argtypes = [ci, i64, i64, vp, i64, vp, i64, vp]
     lib.sp24_compress.argtypes = [ci, i64, i64, vp, i64, vp, i64, vp, ci, vp, vp]
     lib.sp24_decompress.argtypes = [ci, i64, i64, vp, i64, vp, ci, vp, i64, vp]
+    lib.sp24_prune_compress.argtypes = [ci, i64, i64, vp, i64, vp, i64, vp, i64, vp, ci, vp, vp]
     lib.sp24_gemm_workspace_bytes.argtypes = [ctypes.POINTER(GemmDesc)]
     lib.sp24_gemm_workspace_bytes.restype = sz
     lib.sp24_gemm.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -154,6 +155,22 @@ def compress_into(x, vals, meta, layout: int = META_TCGEN05, dtype: str | None =
     _check(lib.sp24_compress(DTYPE_CODE[dt], M, K, _ptr(x), x.stride(0) if M > 1 else K, _ptr(vals),
                              vals.stride(0) if M > 1 else K // 2, _ptr(meta), layout, _ptr(dropped),
                              _stream()), "sp24_compress")
+
+
+def prune_compress(x: torch.Tensor, layout: int = META_TCGEN05, dtype: str | None = None, count_dropped: bool = False,
+                   pruned: torch.Tensor | None = None, vals: torch.Tensor | None = None,
+                   meta: torch.Tensor | None = None):
+    """sp24_prune_compress: one pass; returns (pruned [M, K], vals [M, K/2], meta, dropped tensor or None)."""
+    dt = _dtype_of(x, dtype)
+    M, K = x.shape
+    pruned = torch.empty_like(x) if pruned is None else pruned
+    vals = torch.empty((M, K // 2), dtype=x.dtype, device=x.device) if vals is None else vals
+    meta = torch.empty(meta_bytes(dt, M, K, layout), dtype=torch.uint8, device=x.device) if meta is None else meta
+    dropped = torch.zeros(1, dtype=torch.int64, device=x.device) if count_dropped else None
+    _check(lib.sp24_prune_compress(DTYPE_CODE[dt], M, K, _ptr(x), x.stride(0) if M > 1 else K, _ptr(pruned),
+                                   pruned.stride(0) if M > 1 else K, _ptr(vals), vals.stride(0) if M > 1 else K // 2,
+                                   _ptr(meta), layout, _ptr(dropped), _stream()), "sp24_prune_compress")
+    return pruned, vals, meta, dropped
 
 
 def decompress(vals: torch.Tensor, meta: torch.Tensor, layout: int = META_TCGEN05,

@@ -221,13 +221,21 @@ __device__ __forceinline__ void count_dropped(uint32_t lost, unsigned long long*
 // 2j+1 hold the two halves of a 16-column chunk; the even lane stores the chunk's 16 metadata bits.
 // HW: metadata goes straight into the tensor-core operand order.  FULL: the launch covers exactly
 // the matrix (no padding rows / columns, no ragged block), so no bounds are checked.
-template <int UNROLL, bool COUNT, bool HW, bool FULL>
-__global__ void __launch_bounds__(kThreads, 4) compress16_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
+// PRUNE: the pruned matrix is written as well (y, same shape as x; may be x itself), so that one
+// pass over x yields everything the separate prune and compress passes would.
+template <int UNROLL, bool COUNT, bool HW, bool FULL, bool PRUNE>
+__global__ void __launch_bounds__(kThreads, 4) compress16_kernel(const uint8_t* x, int64_t row_bytes_x,
                                                               uint8_t* __restrict__ vals, int64_t row_bytes_v,
                                                               uint8_t* __restrict__ meta, int64_t M, int64_t K,
                                                               int64_t rows_pad, int64_t chunks_pad,
-                                                              unsigned long long* dropped) {
+                                                              unsigned long long* dropped, uint8_t* y,
+                                                              int64_t row_bytes_y) {
   __shared__ uint32_t table[64];
+  __shared__ uint32_t ptable[PRUNE ? 64 : 1];
+  if (PRUNE) {
+    const int t = threadIdx.y * blockDim.x + threadIdx.x;
+    if (t < 64) ptable[t] = prune_selectors<2>((uint32_t)t);
+  }
   build_selection_table(table);
   const uint32_t halves = (uint32_t)(K >> 3), halves_pad = (uint32_t)chunks_pad * 2, KB = (uint32_t)(chunks_pad >> 3);
   const uint32_t h0 = blockIdx.x * UNROLL * blockDim.x + threadIdx.x;
@@ -259,8 +267,15 @@ __global__ void __launch_bounds__(kThreads, 4) compress16_kernel(const uint8_t* 
       uint32_t mbyte = 0x44u;  // padding: positions (0, 1) in both groups
       if (row_live && (FULL || half < halves)) {
         const uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
-        const uint32_t e0 = table[selection_index(w[0] & 0x7FFF7FFFu, w[1] & 0x7FFF7FFFu)];
-        const uint32_t e1 = table[selection_index(w[2] & 0x7FFF7FFFu, w[3] & 0x7FFF7FFFu)];
+        const uint32_t i0 = selection_index(w[0] & 0x7FFF7FFFu, w[1] & 0x7FFF7FFFu);
+        const uint32_t i1 = selection_index(w[2] & 0x7FFF7FFFu, w[3] & 0x7FFF7FFFu);
+        const uint32_t e0 = table[i0], e1 = table[i1];
+        if (PRUNE) {
+          const uint32_t s0 = ptable[i0], s1 = ptable[i1];
+          st_stream(y + row * row_bytes_y + half * 16u,
+                    make_uint4(__byte_perm(w[0], 0, s0 & 0xFFFFu), __byte_perm(w[1], 0, s0 >> 16),
+                               __byte_perm(w[2], 0, s1 & 0xFFFFu), __byte_perm(w[3], 0, s1 >> 16)));
+        }
         __stcs(reinterpret_cast<uint2*>(vr + half * 8u),
                make_uint2(__byte_perm(w[0], w[1], e0 >> 16), __byte_perm(w[2], w[3], e1 >> 16)));
         mbyte = (e0 & 0xFu) | ((e1 & 0xFu) << 4);
@@ -278,13 +293,19 @@ __global__ void __launch_bounds__(kThreads, 4) compress16_kernel(const uint8_t* 
 
 // int8.  Work unit: one chunk of 16 columns (four groups) = one 16-byte load, 8 bytes of values and
 // 16 bits of metadata out.
-template <int UNROLL, bool COUNT, bool HW, bool FULL>
-__global__ void __launch_bounds__(kThreads, 4) compress8_kernel(const uint8_t* __restrict__ x, int64_t row_bytes_x,
+template <int UNROLL, bool COUNT, bool HW, bool FULL, bool PRUNE>
+__global__ void __launch_bounds__(kThreads, 4) compress8_kernel(const uint8_t* x, int64_t row_bytes_x,
                                                              uint8_t* __restrict__ vals, int64_t row_bytes_v,
                                                              uint8_t* __restrict__ meta, int64_t M, int64_t K,
                                                              int64_t rows_pad, int64_t chunks_pad,
-                                                             unsigned long long* dropped, int f8) {
+                                                             unsigned long long* dropped, int f8, uint8_t* y,
+                                                             int64_t row_bytes_y) {
   __shared__ uint32_t table[64];
+  __shared__ uint32_t ptable[PRUNE ? 64 : 1];
+  if (PRUNE) {
+    const int t = threadIdx.y * blockDim.x + threadIdx.x;
+    if (t < 64) ptable[t] = prune_selectors<1>((uint32_t)t);
+  }
   build_selection_table(table);
   const uint32_t chunks = (uint32_t)(K >> 4), cpad = (uint32_t)chunks_pad, KB = (uint32_t)(chunks_pad >> 3);
   const uint32_t c0 = blockIdx.x * UNROLL * blockDim.x + threadIdx.x;
@@ -315,17 +336,21 @@ __global__ void __launch_bounds__(kThreads, 4) compress8_kernel(const uint8_t* _
       if (row_live && (FULL || chunk < chunks)) {
         const uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
         uint32_t out[2] = {0, 0};
+        uint32_t pw[4];
         mbits = 0;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           const uint32_t a = keys8(w[g], f8);
-          const uint32_t e = table[selection_index(__byte_perm(a, 0, 0x4140), __byte_perm(a, 0, 0x4342))];
+          const uint32_t idx = selection_index(__byte_perm(a, 0, 0x4140), __byte_perm(a, 0, 0x4342));
+          const uint32_t e = table[idx];
+          if (PRUNE) pw[g] = __byte_perm(w[g], 0, ptable[idx]);
           const uint32_t pair = __byte_perm(w[g], 0, ((e >> 8) & 0xFFu) | 0x4400u);
           out[g >> 1] |= pair << (16 * (g & 1));
           mbits |= (e & 0xFu) << (4 * g);
           if (COUNT) lost += __popc(Group8::nonzero(a) & ~(e >> 4) & 0xFu);
         }
         __stcs(reinterpret_cast<uint2*>(vr + chunk * 8u), make_uint2(out[0], out[1]));
+        if (PRUNE) st_stream(y + row * row_bytes_y + chunk * 16u, make_uint4(pw[0], pw[1], pw[2], pw[3]));
       }
       *reinterpret_cast<uint16_t*>(mr + moff[u]) = (uint16_t)mbits;
     }
@@ -633,6 +658,98 @@ extern "C" sp24_status sp24_prune(sp24_dtype t, int64_t M, int64_t K, const void
   return cuda_status(cudaGetLastError());
 }
 
+namespace sp24 {
+namespace {
+
+template <int ES, bool COUNT, bool HW, bool FULL, bool PRUNE>
+void launch_compress_vec(const RowLaunch& L, cudaStream_t s, const uint8_t* xs, int64_t rbx, uint8_t* vs, int64_t rbv,
+                         uint8_t* ms, int64_t M, int64_t K, int64_t rows_pad, int64_t chunks_pad,
+                         unsigned long long* dropped, int f8, uint8_t* ys, int64_t rby) {
+  constexpr int UNROLL = 4;
+  if (ES == 2)
+    compress16_kernel<UNROLL, COUNT, HW, FULL, PRUNE><<<L.grid, L.block, 0, s>>>(xs, rbx, vs, rbv, ms, M, K, rows_pad,
+                                                                                chunks_pad, dropped, ys, rby);
+  else
+    compress8_kernel<UNROLL, COUNT, HW, FULL, PRUNE><<<L.grid, L.block, 0, s>>>(xs, rbx, vs, rbv, ms, M, K, rows_pad,
+                                                                               chunks_pad, dropped, f8, ys, rby);
+}
+
+// compress (y == nullptr) or fused prune + compress (y = pruned matrix, vector kernels only: returns
+// SP24_ERR_UNSUPPORTED when they cannot take the operands) for the 2:4 types.
+sp24_status compress_any(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx, void* y, int64_t ldy,
+                         void* vals, int64_t ldv, void* meta, sp24_meta_layout l, unsigned long long* dropped,
+                         void* stream) {
+  sp24_status st = validate_matrix_args(t, M, K, 8);
+  if (st != SP24_OK) return st;
+  SP24_RETURN_IF(l != SP24_META_CANONICAL && l != SP24_META_TCGEN05, SP24_ERR_UNSUPPORTED);
+  if (M == 0 || K == 0) return SP24_OK;
+  SP24_RETURN_IF(x == nullptr || vals == nullptr || meta == nullptr, SP24_ERR_NULL);
+  SP24_RETURN_IF(ldx < K || ldv < K / 2, SP24_ERR_STRIDE);
+  if ((st = check_arch()) != SP24_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int es = elem_bytes(t), f8 = is_fp8(t) ? 1 : 0;
+  const bool hw = l == SP24_META_TCGEN05;
+  const int64_t rows_pad = hw ? (M + 127) / 128 * 128 : M;
+  const int64_t k_pad = hw ? (K + 255) / 256 * 256 : K;
+  const bool vec = K % 16 == 0 && aligned16(x) && aligned16(vals) && aligned16(meta) && (ldx * es) % 16 == 0 &&
+                   (ldv * es) % (8 * es) == 0;
+  if (vec) {
+    constexpr int UNROLL = 4;
+    const int64_t chunks_pad = k_pad / 16;
+    const int64_t units = es == 2 ? chunks_pad * 2 : chunks_pad;  // 16-byte vectors per padded row
+    RowLaunch L(units, rows_pad, UNROLL);
+    const bool full = rows_pad == M && k_pad == K && units % ((int64_t)L.block.x * UNROLL) == 0;
+    const int variant = (y ? 8 : 0) | (dropped ? 4 : 0) | (hw ? 2 : 0) | (full ? 1 : 0);
+    const uint8_t* xs = (const uint8_t*)x;
+    uint8_t *vs = (uint8_t*)vals, *ms = (uint8_t*)meta, *ys = (uint8_t*)y;
+#define SP24_CV(V, COUNT, HW, FULL, PRUNE)                                                                            \
+  case V:                                                                                                             \
+    if (es == 2)                                                                                                      \
+      launch_compress_vec<2, COUNT, HW, FULL, PRUNE>(L, s, xs, ldx * es, vs, ldv * es, ms, M, K, rows_pad, chunks_pad, \
+                                                     dropped, f8, ys, ldy * es);                                      \
+    else                                                                                                              \
+      launch_compress_vec<1, COUNT, HW, FULL, PRUNE>(L, s, xs, ldx * es, vs, ldv * es, ms, M, K, rows_pad, chunks_pad, \
+                                                     dropped, f8, ys, ldy * es);                                      \
+    break;
+    switch (variant) {
+      SP24_CV(0, false, false, false, false)
+      SP24_CV(1, false, false, true, false)
+      SP24_CV(2, false, true, false, false)
+      SP24_CV(3, false, true, true, false)
+      SP24_CV(4, true, false, false, false)
+      SP24_CV(5, true, false, true, false)
+      SP24_CV(6, true, true, false, false)
+      SP24_CV(7, true, true, true, false)
+      SP24_CV(8, false, false, false, true)
+      SP24_CV(9, false, false, true, true)
+      SP24_CV(10, false, true, false, true)
+      SP24_CV(11, false, true, true, true)
+      SP24_CV(12, true, false, false, true)
+      SP24_CV(13, true, false, true, true)
+      SP24_CV(14, true, true, false, true)
+      default:
+        SP24_CV(15, true, true, true, true)
+    }
+#undef SP24_CV
+  } else {
+    if (y != nullptr) return SP24_ERR_UNSUPPORTED;
+    int64_t bytes_pad = k_pad / 8, total = rows_pad * bytes_pad;
+    unsigned blocks = blocks_for(total, kThreads);
+    if (es == 2)
+      compress_scalar_kernel<uint16_t><<<blocks, kThreads, 0, s>>>((const uint16_t*)x, ldx, (uint16_t*)vals, ldv,
+                                                                   (uint8_t*)meta, (int)l, M, K, rows_pad, bytes_pad,
+                                                                   dropped, 0);
+    else
+      compress_scalar_kernel<int8_t><<<blocks, kThreads, 0, s>>>((const int8_t*)x, ldx, (int8_t*)vals, ldv,
+                                                                 (uint8_t*)meta, (int)l, M, K, rows_pad, bytes_pad,
+                                                                 dropped, f8);
+  }
+  return cuda_status(cudaGetLastError());
+}
+
+}  // namespace
+}  // namespace sp24
+
 extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx, void* vals,
                                      int64_t ldv, void* meta, sp24_meta_layout l, unsigned long long* dropped,
                                      void* stream) {
@@ -657,76 +774,23 @@ extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const v
                                                         M, K, rows_pad, k_pad / 8, dropped);
     return cuda_status(cudaGetLastError());
   }
-  sp24_status st = validate_matrix_args(t, M, K, 8);
-  if (st != SP24_OK) return st;
-  SP24_RETURN_IF(l != SP24_META_CANONICAL && l != SP24_META_TCGEN05, SP24_ERR_UNSUPPORTED);
-  if (M == 0 || K == 0) return SP24_OK;
-  SP24_RETURN_IF(x == nullptr || vals == nullptr || meta == nullptr, SP24_ERR_NULL);
-  SP24_RETURN_IF(ldx < K || ldv < K / 2, SP24_ERR_STRIDE);
-  if ((st = check_arch()) != SP24_OK) return st;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const int es = elem_bytes(t), f8 = is_fp8(t) ? 1 : 0;
-  const bool hw = l == SP24_META_TCGEN05;
-  const int64_t rows_pad = hw ? (M + 127) / 128 * 128 : M;
-  const int64_t k_pad = hw ? (K + 255) / 256 * 256 : K;
-  const bool vec = K % 16 == 0 && aligned16(x) && aligned16(vals) && aligned16(meta) && (ldx * es) % 16 == 0 &&
-                   (ldv * es) % (8 * es) == 0;
-  if (vec) {
-    constexpr int UNROLL = 4;
-    int64_t chunks_pad = k_pad / 16;
-    const uint8_t* xs = (const uint8_t*)x;
-    uint8_t *vs = (uint8_t*)vals, *ms = (uint8_t*)meta;
-    if (es == 2) {
-      RowLaunch L(chunks_pad * 2, rows_pad, UNROLL);
-      const bool full = rows_pad == M && k_pad == K &&
-                        (chunks_pad * 2) % ((int64_t)L.block.x * UNROLL) == 0;
-      const int variant = (dropped ? 4 : 0) | (hw ? 2 : 0) | (full ? 1 : 0);
-#define SP24_C16(COUNT, HW, FULL)                                                                          \
-  compress16_kernel<UNROLL, COUNT, HW, FULL><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, M, K, \
-                                                                        rows_pad, chunks_pad, dropped)
-      switch (variant) {
-        case 0: SP24_C16(false, false, false); break;
-        case 1: SP24_C16(false, false, true); break;
-        case 2: SP24_C16(false, true, false); break;
-        case 3: SP24_C16(false, true, true); break;
-        case 4: SP24_C16(true, false, false); break;
-        case 5: SP24_C16(true, false, true); break;
-        case 6: SP24_C16(true, true, false); break;
-        default: SP24_C16(true, true, true); break;
-      }
-#undef SP24_C16
-    } else {
-      RowLaunch L(chunks_pad, rows_pad, UNROLL);
-      const bool full = rows_pad == M && k_pad == K && chunks_pad % ((int64_t)L.block.x * UNROLL) == 0;
-      const int variant = (dropped ? 4 : 0) | (hw ? 2 : 0) | (full ? 1 : 0);
-#define SP24_C8(COUNT, HW, FULL)                                                                          \
-  compress8_kernel<UNROLL, COUNT, HW, FULL><<<L.grid, L.block, 0, s>>>(xs, ldx * es, vs, ldv * es, ms, M, K, \
-                                                                       rows_pad, chunks_pad, dropped, f8)
-      switch (variant) {
-        case 0: SP24_C8(false, false, false); break;
-        case 1: SP24_C8(false, false, true); break;
-        case 2: SP24_C8(false, true, false); break;
-        case 3: SP24_C8(false, true, true); break;
-        case 4: SP24_C8(true, false, false); break;
-        case 5: SP24_C8(true, false, true); break;
-        case 6: SP24_C8(true, true, false); break;
-        default: SP24_C8(true, true, true); break;
-      }
-#undef SP24_C8
-    }
-  } else {
-    int64_t bytes_pad = k_pad / 8, total = rows_pad * bytes_pad;
-    unsigned blocks = blocks_for(total, kThreads);
-    if (es == 2)
-      compress_scalar_kernel<uint16_t><<<blocks, kThreads, 0, s>>>((const uint16_t*)x, ldx, (uint16_t*)vals, ldv,
-                                                                   (uint8_t*)meta, (int)l, M, K, rows_pad, bytes_pad,
-                                                                   dropped, 0);
-    else
-      compress_scalar_kernel<int8_t><<<blocks, kThreads, 0, s>>>((const int8_t*)x, ldx, (int8_t*)vals, ldv,
-                                                                 (uint8_t*)meta, (int)l, M, K, rows_pad, bytes_pad,
-                                                                 dropped, f8);
+  return compress_any(t, M, K, x, ldx, nullptr, 0, vals, ldv, meta, l, dropped, stream);
+}
+
+extern "C" sp24_status sp24_prune_compress(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx, void* y,
+                                           int64_t ldy, void* vals, int64_t ldv, void* meta, sp24_meta_layout l,
+                                           unsigned long long* dropped, void* stream) {
+  const int es = elem_bytes(t);
+  const bool fused = is_ab_type(t) && y != nullptr && aligned16(y) && es > 0 && (ldy * es) % 16 == 0 && ldy >= K;
+  if (fused) {
+    const sp24_status st = compress_any(t, M, K, x, ldx, y, ldy, vals, ldv, meta, l, dropped, stream);
+    if (st != SP24_ERR_UNSUPPORTED) return st;
   }
-  return cuda_status(cudaGetLastError());
+  // no fused kernel for this case (1:2 pattern, or operands the vector kernels cannot take): two passes.
+  // compress reads x before prune may overwrite it (y may be x).
+  sp24_status st = sp24_compress(t, M, K, x, ldx, vals, ldv, meta, l, dropped, stream);
+  if (st != SP24_OK) return st;
+  return sp24_prune(t, M, K, x, ldx, y, ldy, stream);
 }
 
 extern "C" sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals, int64_t ldv,

@@ -113,3 +113,43 @@ def test_im2col_bit_exact(sp, dtype):
     got = sp.im2col_nhwc_3x3(to_device(x, dtype))
     assert np.array_equal(to_host_bits(got), oracle.im2col_nhwc_3x3(x, dtype))
     assert got.shape == (cfg.N, cfg.K)
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16", "i8"])
+@pytest.mark.parametrize("shape", [(128, 256), (200, 336), (37, 96), (513, 1040), (1024, 4096)])
+@pytest.mark.parametrize("layout", [0, 1])
+def test_fused_prune_compress_equals_the_two_passes(sp, dtype, shape, layout):
+    """sp24_prune_compress: one pass over x gives prune(x) and compress(x) bit for bit (oracle on both),
+    also in place (y = x) and with the dropped count."""
+    M, K = shape
+    cfg = inputs.scaled(inputs.CONFIGS["int8_linear" if dtype == "i8" else "tiny_f16"], M=M, N=32, K=K)
+    x = inputs._matrix(cfg.a_dist, dtype, 77, inputs.TENSOR_A, K, 0, M)
+    x[::3, ::5] = 0
+    xd = to_device(x, dtype)
+    pruned, vals, meta, dropped = sp.prune_compress(xd, layout=layout, count_dropped=True)
+    v_ref, m_ref, d_ref = oracle.compress(x, dtype)
+    assert np.array_equal(to_host_bits(pruned), oracle.prune(x, dtype))
+    assert np.array_equal(to_host_bits(vals), v_ref)
+    expect = m_ref.ravel() if layout == 0 else oracle.meta_to_operand_order(m_ref, dtype)
+    assert np.array_equal(meta.cpu().numpy(), expect)
+    assert int(dropped.item()) == d_ref
+    inplace = xd.clone()
+    p2, v2, m2, _ = sp.prune_compress(inplace, layout=layout, pruned=inplace)
+    assert p2.data_ptr() == inplace.data_ptr()
+    assert torch.equal(inplace.view(torch.uint8), pruned.view(torch.uint8))
+    assert torch.equal(v2.view(torch.uint8), vals.view(torch.uint8)) and torch.equal(m2, meta)
+
+
+def test_fused_prune_compress_falls_back_for_unaligned_operands(sp):
+    """An odd leading dimension takes the element-wise kernels (two passes) with the same result."""
+    M, K, ld = 64, 96, 99
+    x = inputs._matrix(("normal", 1.0), "bf16", 78, inputs.TENSOR_A, K, 0, M)
+    buf = torch.zeros(M, ld, dtype=torch.bfloat16, device="cuda")
+    buf[:, :K] = to_device(x, "bf16")
+    xd = buf[:, :K]
+    out = torch.zeros(M, ld, dtype=torch.bfloat16, device="cuda")[:, :K]
+    pruned, vals, meta, _ = sp.prune_compress(xd, layout=0, pruned=out)
+    v_ref, m_ref, _ = oracle.compress(x, "bf16")
+    assert np.array_equal(to_host_bits(pruned.contiguous()), oracle.prune(x, "bf16"))
+    assert np.array_equal(to_host_bits(vals), v_ref)
+    assert np.array_equal(meta.cpu().numpy(), m_ref.ravel())

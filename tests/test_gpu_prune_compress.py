@@ -153,3 +153,38 @@ def test_fused_prune_compress_falls_back_for_unaligned_operands(sp):
     assert np.array_equal(to_host_bits(pruned.contiguous()), oracle.prune(x, "bf16"))
     assert np.array_equal(to_host_bits(vals), v_ref)
     assert np.array_equal(meta.cpu().numpy(), m_ref.ravel())
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16", "i8"])
+def test_every_bit_pattern_in_every_position(sp, dtype):
+    """All 65536 (256 for int8) encodings -- zeros of both signs, subnormals, infinities and NaN
+    patterns, -128 -- meet random partners in every position of a group: prune, compress (both
+    layouts) and the fused pass against the oracle, bit for bit."""
+    rng = np.random.default_rng(5)
+    n = 256 if dtype == "i8" else 65536
+    store = np.int8 if dtype == "i8" else np.uint16
+    allv = np.arange(n, dtype=np.uint8 if dtype == "i8" else np.uint16).view(store)
+    M, K = 4 * n // 256, 1024                       # every pattern once in each of the four positions
+    x = rng.integers(0, n, size=(M, K)).astype(np.uint16 if dtype != "i8" else np.uint8).view(store)
+    x = np.ascontiguousarray(x)
+    groups = x.reshape(-1, 4)
+    for pos in range(4):
+        groups[pos * n:(pos + 1) * n, pos] = allv      # group pos*n + v holds pattern v at position pos
+    # near-ties: copy the pattern into a second position with the sign flipped in a quarter of the groups
+    flip = np.uint16(0x8000) if dtype != "i8" else None
+    if flip is not None:
+        g16 = groups.view(np.uint16)
+        g16[::4, 3] = g16[::4, 0] ^ flip
+    x = groups.reshape(M, K)
+    xd = to_device(x, dtype)
+    assert np.array_equal(to_host_bits(sp.prune(xd)), oracle.prune(x, dtype))
+    v_ref, m_ref, d_ref = oracle.compress(x, dtype)
+    for layout in (0, 1):
+        vals, meta, dropped = sp.compress(xd, layout=layout, count_dropped=True)
+        assert np.array_equal(to_host_bits(vals), v_ref)
+        expect = m_ref.ravel() if layout == 0 else oracle.meta_to_operand_order(m_ref, dtype)
+        assert np.array_equal(meta.cpu().numpy(), expect)
+        assert int(dropped.item()) == d_ref
+    pruned, vals, meta, _ = sp.prune_compress(xd, layout=1)
+    assert np.array_equal(to_host_bits(pruned), oracle.prune(x, dtype))
+    assert np.array_equal(to_host_bits(vals), v_ref)

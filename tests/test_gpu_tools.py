@@ -55,3 +55,39 @@ def test_prune_2d(sp, dtype):
     assert np.array_equal(to_host_bits(y), oracle.prune_2d(x, dtype))
     with pytest.raises(sp.Sp24Error):
         sp.prune_2d(to_device(x[:130], dtype))                           # M % 4 != 0
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", [(64, 512), (37, 4096), (5, 32768), (130, 264)])
+def test_kept_magnitude_vector_and_scalar_paths(sp, dtype, shape):
+    """Rows that take the 16-byte-vector kernels, rows too long for the shared-memory gather of the
+    permuted form (32768 16-bit columns), and an unaligned view that takes the element-wise kernel."""
+    M, K = shape
+    x = _rand(dtype, M, K, 6)
+    x[::2, ::3] = 0
+    perm = np.random.default_rng(2).permutation(K).astype(np.int32)
+    permd = torch.from_numpy(perm).cuda()
+    want, want_p = oracle.kept_magnitude(x, dtype), oracle.kept_magnitude(x, dtype, perm)
+    xd = to_device(x, dtype)
+    assert abs(float(sp.kept_magnitude(xd).item()) - want) <= 1e-12 * want
+    assert abs(float(sp.kept_magnitude(xd, permd).item()) - want_p) <= 1e-12 * want_p
+    wide = torch.zeros(M, K + 3, dtype=xd.dtype, device="cuda")           # odd leading dimension
+    wide[:, :K] = xd
+    view = wide[:, :K]
+    assert abs(float(sp.kept_magnitude(view).item()) - want) <= 1e-12 * want
+    assert abs(float(sp.kept_magnitude(view, permd).item()) - want_p) <= 1e-12 * want_p
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_apply_mask_and_prune_2d_on_unaligned_views(sp, dtype):
+    M, K = 68, 264
+    x, w = _rand(dtype, M, K, 7), _rand(dtype, M, K, 8)
+    _, meta_ref, _ = oracle.compress(x, dtype)
+    _, meta, _ = sp.compress(to_device(x, dtype), layout=0)
+    wide = torch.zeros(M, K + 5, dtype=to_device(w, dtype).dtype, device="cuda")
+    wide[:, :K] = to_device(w, dtype)
+    view = wide[:, :K]
+    assert np.array_equal(to_host_bits(sp.apply_mask(view, meta, layout=0).contiguous()), oracle.apply_mask(w, meta_ref, dtype))
+    assert np.array_equal(to_host_bits(sp.prune_2d(view).contiguous()), oracle.prune_2d(w, dtype))
+    big = _rand(dtype, 512, 2048, 9)
+    assert np.array_equal(to_host_bits(sp.prune_2d(to_device(big, dtype))), oracle.prune_2d(big, dtype))

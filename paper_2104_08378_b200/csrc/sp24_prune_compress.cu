@@ -455,26 +455,29 @@ __global__ void decompress_scalar_kernel(const T* __restrict__ vals, int64_t ldv
 }
 
 // ---- im2col (3x3, stride 1, pad 1, NHWC) ------------------------------------------------------
-// One 16-byte vector of the output per thread: out row = output pixel, out column = (r, s, c).
-__global__ void __launch_bounds__(kThreads) im2col_3x3_kernel(const uint8_t* __restrict__ in, uint8_t* __restrict__ out,
-                                                              int64_t row_bytes_out, int H, int W, int64_t c_vecs,
-                                                              int64_t total) {
-  int64_t id = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-  if (id >= total) return;
-  int64_t vec_per_pixel = 9 * c_vecs;
-  int64_t pixel = id / vec_per_pixel, rem = id - pixel * vec_per_pixel;
-  int rs = (int)(rem / c_vecs);
-  int64_t cv = rem - rs * c_vecs;
-  int r = rs / 3, s = rs - 3 * r;
-  int w = (int)(pixel % W);
-  int64_t t = pixel / W;
-  int h = (int)(t % H);
-  int64_t n = t / H;
-  int hh = h + r - 1, ww = w + s - 1;
-  uint4 v = make_uint4(0, 0, 0, 0);
-  if (hh >= 0 && hh < H && ww >= 0 && ww < W)
-    v = __ldg(reinterpret_cast<const uint4*>(in + (((n * H + hh) * W + ww) * c_vecs + cv) * 16));
-  st_stream(out + pixel * row_bytes_out + rem * 16, v);
+// Out row = output pixel, out column = (r, s, c).  A block handles the pixels of one image row (n, h):
+// blockIdx.x = h, blockIdx.y strides over n, threadIdx = (16-byte vector of channels, filter tap, pixel
+// column), so no thread divides anything and a warp writes 512 contiguous bytes.
+__global__ void __launch_bounds__(kThreads + 64) im2col_3x3_kernel(const uint8_t* __restrict__ in, uint8_t* __restrict__ out,
+                                                                   int64_t row_bytes_out, int64_t Nb, int H, int W,
+                                                                   int c_vecs) {
+  const int h = blockIdx.x, rs = threadIdx.y, r = rs / 3, s = rs - 3 * r;
+  const int hh = h + r - 1;
+  const bool row_ok = hh >= 0 && hh < H;
+  for (int64_t n = blockIdx.y; n < Nb; n += gridDim.y) {
+    const uint8_t* in_row = in + ((n * H + hh) * W) * (int64_t)c_vecs * 16;
+    uint8_t* out_row = out + ((n * H + h) * W) * row_bytes_out + (int64_t)rs * c_vecs * 16;
+#pragma unroll 4
+    for (int w = threadIdx.z; w < W; w += blockDim.z) {
+      const int ww = w + s - 1;
+      const bool ok = row_ok && ww >= 0 && ww < W;
+      for (int cv = threadIdx.x; cv < c_vecs; cv += blockDim.x) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (ok) v = __ldg(reinterpret_cast<const uint4*>(in_row + ((int64_t)ww * c_vecs + cv) * 16));
+        st_stream(out_row + w * row_bytes_out + cv * 16, v);
+      }
+    }
+  }
 }
 
 // ---- the 1:2 pattern of the TF32 mode (Section 3.2): fp32 storage, one kept value per aligned pair ----
@@ -863,8 +866,13 @@ extern "C" sp24_status sp24_im2col_nhwc_3x3(sp24_dtype t, int64_t Nb, int64_t H,
   SP24_RETURN_IF(!aligned16(in) || !aligned16(out), SP24_ERR_ALIGN);
   sp24_status st = check_arch();
   if (st != SP24_OK) return st;
-  int64_t c_vecs = C * es / 16, total = Nb * H * W * 9 * c_vecs;
-  im2col_3x3_kernel<<<blocks_for(total, kThreads), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      (const uint8_t*)in, (uint8_t*)out, ldo * es, (int)H, (int)W, c_vecs, total);
+  const int64_t c_vecs = C * es / 16;
+  SP24_RETURN_IF(c_vecs > (1 << 24), SP24_ERR_SHAPE);
+  const unsigned bx = (unsigned)(c_vecs < 32 ? c_vecs : 32);
+  unsigned bz = 288u / (9u * bx);
+  bz = bz < 1 ? 1 : (bz > (unsigned)W ? (unsigned)W : bz);
+  const dim3 block(bx, 9, bz), grid((unsigned)H, (unsigned)(Nb < 65535 ? Nb : 65535), 1);
+  im2col_3x3_kernel<<<grid, block, 0, static_cast<cudaStream_t>(stream)>>>((const uint8_t*)in, (uint8_t*)out, ldo * es, Nb,
+                                                                           (int)H, (int)W, (int)c_vecs);
   return cuda_status(cudaGetLastError());
 }

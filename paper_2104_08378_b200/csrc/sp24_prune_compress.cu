@@ -133,6 +133,32 @@ __device__ __forceinline__ uint32_t selection_index(uint32_t k_lo, uint32_t k_hi
   return ((t >> 13) & 7u) | ((t >> 26) & 0x38u);
 }
 
+// 8-bit types: the table indices of the four groups of one 16-byte vector at once.  a[g] holds the four
+// keys of group g, one per byte.  With all keys below 128 the keys are transposed (word p = key p of
+// the four groups) and each of the six comparisons is one byte-wise subtraction with a guard bit,
+// ((x | 0x80) - y) bit 7 = (x >= y); the six flag words are merged into one index byte per group.  A
+// key of 128 (int8 -128) does not fit the guard trick: such a vector takes the group-by-group path.
+__device__ __forceinline__ void selection_index_x4(const uint32_t (&a)[4], uint32_t (&idx)[4]) {
+  if ((a[0] | a[1] | a[2] | a[3]) & 0x80808080u) {
+#pragma unroll
+    for (int g = 0; g < 4; ++g) idx[g] = selection_index(__byte_perm(a[g], 0, 0x4140), __byte_perm(a[g], 0, 0x4342));
+    return;
+  }
+  const uint32_t t0 = __byte_perm(a[0], a[1], 0x5140), t1 = __byte_perm(a[2], a[3], 0x5140);
+  const uint32_t t2 = __byte_perm(a[0], a[1], 0x7362), t3 = __byte_perm(a[2], a[3], 0x7362);
+  const uint32_t p0 = __byte_perm(t0, t1, 0x5410), p1 = __byte_perm(t0, t1, 0x7632);
+  const uint32_t p2 = __byte_perm(t2, t3, 0x5410), p3 = __byte_perm(t2, t3, 0x7632);
+  const uint32_t g = 0x80808080u;
+  const uint32_t c01 = ((p0 | g) - p1) & g, c02 = ((p0 | g) - p2) & g, c03 = ((p0 | g) - p3) & g;
+  const uint32_t c12 = ((p1 | g) - p2) & g, c13 = ((p1 | g) - p3) & g, c23 = ((p2 | g) - p3) & g;
+  // index bits: 0 = c01, 1 = c03, 2 = c02, 3 = c23, 4 = c12, 5 = c13 (see selection_entry); byte g of x = group g
+  const uint32_t x = (c01 >> 7) | (c03 >> 6) | (c02 >> 5) | (c23 >> 4) | (c12 >> 3) | (c13 >> 2);
+  idx[0] = x & 0xFFu;
+  idx[1] = (x >> 8) & 0xFFu;
+  idx[2] = (x >> 16) & 0xFFu;
+  idx[3] = x >> 24;
+}
+
 // ---- prune (vectorised) -------------------------------------------------------------------------
 // Launch geometry of the vectorised kernels: blockDim = (TX, 256/TX), a warp always lies inside
 // one row; thread (tx, ty) of block (bx, by) handles units (bx*UNROLL + u)*TX + tx, u < UNROLL, of
@@ -162,11 +188,11 @@ __device__ __forceinline__ uint4 prune_vec(uint4 v, const uint32_t* table, int f
                       __byte_perm(v.w, 0, s1 >> 16));
   }
   uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  const uint32_t a[4] = {keys8(w[0], f8), keys8(w[1], f8), keys8(w[2], f8), keys8(w[3], f8)};
+  uint32_t idx[4];
+  selection_index_x4(a, idx);
 #pragma unroll
-  for (int g = 0; g < 4; ++g) {
-    const uint32_t a = keys8(w[g], f8);
-    w[g] = __byte_perm(w[g], 0, table[selection_index(__byte_perm(a, 0, 0x4140), __byte_perm(a, 0, 0x4342))]);
-  }
+  for (int g = 0; g < 4; ++g) w[g] = __byte_perm(w[g], 0, table[idx[g]]);
   return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
@@ -338,10 +364,13 @@ __global__ void __launch_bounds__(kThreads, 4) compress8_kernel(const uint8_t* x
         uint32_t out[2] = {0, 0};
         uint32_t pw[4];
         mbits = 0;
+        const uint32_t keys[4] = {keys8(w[0], f8), keys8(w[1], f8), keys8(w[2], f8), keys8(w[3], f8)};
+        uint32_t idx4[4];
+        selection_index_x4(keys, idx4);
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-          const uint32_t a = keys8(w[g], f8);
-          const uint32_t idx = selection_index(__byte_perm(a, 0, 0x4140), __byte_perm(a, 0, 0x4342));
+          const uint32_t a = keys[g];
+          const uint32_t idx = idx4[g];
           const uint32_t e = table[idx];
           if (PRUNE) pw[g] = __byte_perm(w[g], 0, ptable[idx]);
           const uint32_t pair = __byte_perm(w[g], 0, ((e >> 8) & 0xFFu) | 0x4400u);
@@ -401,10 +430,11 @@ __global__ void __launch_bounds__(kThreads) decompress_vec_kernel(const uint8_t*
                                                                   const uint8_t* __restrict__ meta, int layout,
                                                                   uint8_t* __restrict__ y, int64_t row_bytes_y,
                                                                   int64_t M, int64_t K, int64_t chunks_pad) {
+  // threads along a row (one 16-column chunk each), blockIdx.y strides over the rows: no division
   const int64_t chunks = K >> 4, KB = chunks_pad >> 3;
-  int64_t id = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-  if (id >= M * chunks) return;
-  int64_t row = id / chunks, chunk = id - row * chunks;
+  const int64_t chunk = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (chunk >= chunks) return;
+  for (int64_t row = blockIdx.y; row < M; row += gridDim.y) {
   uint32_t mbits = *reinterpret_cast<const uint16_t*>(meta + meta_offset<ES>(layout, row, chunk, K, KB));
   if (ES == 2) {
     uint4 v = ld_stream(vals + row * row_bytes_v + chunk * 16);
@@ -431,6 +461,7 @@ __global__ void __launch_bounds__(kThreads) decompress_vec_kernel(const uint8_t*
       w[g] = ((pair & 0xFFu) << (8 * (nib & 3))) | ((pair >> 8) << (8 * (nib >> 2)));
     }
     st_stream(y + row * row_bytes_y + chunk * 16, make_uint4(w[0], w[1], w[2], w[3]));
+  }
   }
 }
 
@@ -833,8 +864,7 @@ extern "C" sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const
   const bool vec = K % 16 == 0 && aligned16(y) && aligned16(vals) && aligned16(meta) && (ldy * es) % 16 == 0 &&
                    (ldv * es) % (8 * es) == 0;
   if (vec) {
-    int64_t total = M * (K / 16);
-    unsigned blocks = blocks_for(total, kThreads);
+    const dim3 blocks((unsigned)((K / 16 + kThreads - 1) / kThreads), (unsigned)(M < 16384 ? M : 16384), 1);
     if (es == 2)
       decompress_vec_kernel<2><<<blocks, kThreads, 0, s>>>((const uint8_t*)vals, ldv * es, (const uint8_t*)meta, (int)l,
                                                            (uint8_t*)y, ldy * es, M, K, k_pad / 16);

@@ -990,7 +990,14 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   const int64_t n_tiles = (d->N + 223) / 224;
   int ctas = 1, block_n = 128, mblk = 1;
   if (d->M >= 512 && (d->M / 512) * n_tiles >= 444) { ctas = 2; block_n = 224; mblk = 2; }
-  else if (d->M >= 256 && (d->M / 256) * n_tiles >= 32) { ctas = 2; block_n = 224; mblk = 1; }
+  else if (d->M >= 256 && (d->M / 256) * n_tiles >= 32) {
+    ctas = 2; block_n = 224; mblk = 1;
+    // Few tokens: every n-tile streams all of A again, so the number of n-tiles decides; 256 columns
+    // (one accumulator buffer, epilogue not overlapped) when that saves one.  Built for the K-contiguous
+    // 16-bit and int8 kinds.
+    const bool has_256 = !tf32 && !f8 && d->order_b == SP24_COL_MAJOR;
+    if (has_256 && d->N <= 2048 && (d->N + 255) / 256 < n_tiles) block_n = 256;
+  }
   p.band = 16 / mblk;
   if (const char* env = getenv("SP24_TILE")) {
     int c = 0, n = 0, m = 1;

@@ -373,9 +373,10 @@ def run_ours(args, cfg):
             opruned = sp.prune(oA)
             oD = torch.empty((oc.M, oc.N), dtype=tdt[oc.cd_type], device=dev)
             s_ms = time_flushed(lambda: sp.gemm(ovals, ometa, oB, out=oD, cd=oc.cd_type, ws=ws))
+            warm_ms = time_call(lambda: sp.gemm(ovals, ometa, oB, out=oD, cd=oc.cd_type, ws=ws))  # operands in the L2
             d_ms = time_flushed(lambda: sp.gemm(opruned, None, oB, out=oD, cd=oc.cd_type, a_is_dense=True, ws=ws))
             peak = 2.0 * peaks["bf16_tflops"] * (2.0 if oc.ab_type == "i8" else 1.0)
-            others[name] = {"M": oc.M, "N": oc.N, "K": oc.K, "ab": oc.ab_type, "gemm_ms": s_ms,
+            others[name] = {"M": oc.M, "N": oc.N, "K": oc.K, "ab": oc.ab_type, "gemm_ms": s_ms, "gemm_l2_warm_ms": warm_ms,
                             "gemm_dense_equiv_tflops": oc.dense_equiv_flop / (s_ms * 1e-3) / 1e12,
                             "frac_of_2x_measured_dense": oc.dense_equiv_flop / (s_ms * 1e-3) / 1e12 / peak,
                             "dense_variant_ms": d_ms, "speedup_vs_dense_variant": d_ms / s_ms}

@@ -1,4 +1,5 @@
 // Size helpers, status strings, the architecture check and the host-buffer pipeline.
+#include <atomic>
 #include <mutex>
 
 #include "sp24_common.cuh"
@@ -6,16 +7,19 @@
 namespace sp24 {
 
 sp24_status check_arch() {
-  static int cached_dev = -1;
-  static sp24_status cached = SP24_ERR_ARCH;
+  // per-device answer: 0 = not asked yet, 1 = sm_100, 2 = something else (callers may be on several threads)
+  static std::atomic<int> known[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SP24_ERR_CUDA;
-  if (dev == cached_dev) return cached;
+  const bool cacheable = dev >= 0 && dev < 64;
+  if (cacheable) {
+    const int k = known[dev].load(std::memory_order_relaxed);
+    if (k != 0) return k == 1 ? SP24_OK : SP24_ERR_ARCH;
+  }
   int major = 0;
   if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SP24_ERR_CUDA;
-  cached_dev = dev;
-  cached = major == 10 ? SP24_OK : SP24_ERR_ARCH;
-  return cached;
+  if (cacheable) known[dev].store(major == 10 ? 1 : 2, std::memory_order_relaxed);
+  return major == 10 ? SP24_OK : SP24_ERR_ARCH;
 }
 
 }  // namespace sp24

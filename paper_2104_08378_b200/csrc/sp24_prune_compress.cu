@@ -133,6 +133,21 @@ __device__ __forceinline__ uint32_t selection_index(uint32_t k_lo, uint32_t k_hi
   return ((t >> 13) & 7u) | ((t >> 26) & 0x38u);
 }
 
+// 16-bit types: the table indices of the two groups of one 16-byte vector at once.  lo/hi are the masked
+// key words of group 0 (k0k1, k2k3) and group 1; word p of the transposed form holds key p of both groups,
+// so each of the six comparisons is one subtraction for the two groups.
+__device__ __forceinline__ void selection_index_x2(uint32_t lo0, uint32_t hi0, uint32_t lo1, uint32_t hi1,
+                                                   uint32_t& idx0, uint32_t& idx1) {
+  const uint32_t p0 = __byte_perm(lo0, lo1, 0x5410), p1 = __byte_perm(lo0, lo1, 0x7632);
+  const uint32_t p2 = __byte_perm(hi0, hi1, 0x5410), p3 = __byte_perm(hi0, hi1, 0x7632);
+  const uint32_t g = 0x80008000u;
+  const uint32_t c01 = ((p0 | g) - p1) & g, c02 = ((p0 | g) - p2) & g, c03 = ((p0 | g) - p3) & g;
+  const uint32_t c12 = ((p1 | g) - p2) & g, c13 = ((p1 | g) - p3) & g, c23 = ((p2 | g) - p3) & g;
+  const uint32_t x = (c01 >> 15) | (c03 >> 14) | (c02 >> 13) | (c23 >> 12) | (c12 >> 11) | (c13 >> 10);
+  idx0 = x & 0xFFFFu;
+  idx1 = x >> 16;
+}
+
 // 8-bit types: the table indices of the four groups of one 16-byte vector at once.  a[g] holds the four
 // keys of group g, one per byte.  With all keys below 128 the keys are transposed (word p = key p of
 // the four groups) and each of the six comparisons is one byte-wise subtraction with a guard bit,
@@ -182,8 +197,9 @@ __device__ __forceinline__ uint32_t prune_selectors(uint32_t idx) {
 template <int ES>
 __device__ __forceinline__ uint4 prune_vec(uint4 v, const uint32_t* table, int f8) {
   if (ES == 2) {
-    const uint32_t s0 = table[selection_index(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu)];
-    const uint32_t s1 = table[selection_index(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu)];
+    uint32_t i0, i1;
+    selection_index_x2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu, v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu, i0, i1);
+    const uint32_t s0 = table[i0], s1 = table[i1];
     return make_uint4(__byte_perm(v.x, 0, s0 & 0xFFFFu), __byte_perm(v.y, 0, s0 >> 16), __byte_perm(v.z, 0, s1 & 0xFFFFu),
                       __byte_perm(v.w, 0, s1 >> 16));
   }
@@ -293,8 +309,8 @@ __global__ void __launch_bounds__(kThreads, 4) compress16_kernel(const uint8_t* 
       uint32_t mbyte = 0x44u;  // padding: positions (0, 1) in both groups
       if (row_live && (FULL || half < halves)) {
         const uint32_t w[4] = {in[u].x, in[u].y, in[u].z, in[u].w};
-        const uint32_t i0 = selection_index(w[0] & 0x7FFF7FFFu, w[1] & 0x7FFF7FFFu);
-        const uint32_t i1 = selection_index(w[2] & 0x7FFF7FFFu, w[3] & 0x7FFF7FFFu);
+        uint32_t i0, i1;
+        selection_index_x2(w[0] & 0x7FFF7FFFu, w[1] & 0x7FFF7FFFu, w[2] & 0x7FFF7FFFu, w[3] & 0x7FFF7FFFu, i0, i1);
         const uint32_t e0 = table[i0], e1 = table[i1];
         if (PRUNE) {
           const uint32_t s0 = ptable[i0], s1 = ptable[i1];

@@ -320,7 +320,7 @@ def run_ours(args, cfg):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / n
 
-    if world == 1 and not args.rows:
+    if world == 1 and not args.rows and not args.no_sustained:
         sus_ms = time_sustained(lambda: sp.gemm(vals, meta, Bt, alpha=cfg.alpha, beta=cfg.beta, C=C, out=Dout, cd=cd, ws=ws))
         kernels["gemm_sustained_ms"] = sus_ms
         kernels["gemm_sustained_dense_equiv_tflops"] = flop / (sus_ms * 1e-3) / 1e12
@@ -503,6 +503,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-other-configs", action="store_true", help="skip the GEMM timings of the other configurations")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the one-second sustained GEMM loops")
     ap.add_argument("--rows", type=int, default=0,
                     help="use only the first ROWS rows of A (a smaller case of the same kernel for ncu captures)")
     args = ap.parse_args()

@@ -184,6 +184,8 @@ def run_reference(args, cfg):
 # -------------------------------------------------------------------------------------------
 def run_ours(args, cfg):
     import torch
+    from paper_2104_08378_b200 import build
+    build.build_library()          # no-op when libsp24.so is newer than its sources; there is no fallback
     from paper_2104_08378_b200 import binding as sp
     from paper_2104_08378_b200 import distributed as D
 

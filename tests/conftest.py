@@ -24,3 +24,16 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """The GPU tests call the in-tree CUDA library: compile it first if it is missing or older than its
+    sources (needs nvcc; without it the tests that need the library fail loudly, there is no fallback)."""
+    try:
+        from paper_2104_08378_b200 import build
+        if build.needs_build():
+            build.build_library()
+    except Exception as e:  # noqa: BLE001 - reported by the tests that need the library
+        print(f"could not build libsp24.so: {e}", file=sys.stderr)
+    yield

@@ -184,14 +184,14 @@ size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d);
  *   A:    device; vals (M x K/2) or dense A (M x K), row-major, 16-byte aligned.
  *   meta: device; TCGEN05-layout metadata of A (ignored when a_is_dense).
  *   B, C, D: device, 16-byte aligned.  C may be NULL iff beta == 0.  C may alias D.
- * The tile shape is chosen from the problem size.  For benchmarking the environment variables
- * SP24_TILE=<CTAs per tile: 1|2>x<columns per tile>x<128-row blocks per CTA: 1|2> (one of the
- * built shapes, else SP24_ERR_UNSUPPORTED) and SP24_BAND=<m-tiles per band of the tile sweep>
- * override the choice; they are read on every call.
  *   workspace: device, >= sp24_gemm_workspace_bytes(d).  The kernel writes a status record
  *              there; read it back with sp24_gemm_status after synchronising.
  * Accumulation is FP32 (INT32) in hardware order; the result is rounded to cd_type once,
- * round-to-nearest-even. */
+ * round-to-nearest-even.
+ * The tile shape is chosen from the problem size.  For benchmarking the environment variables
+ * SP24_TILE=<CTAs per tile: 1|2>x<columns per tile>x<128-row blocks per CTA: 1|2> (one of the
+ * built shapes, else SP24_ERR_UNSUPPORTED) and SP24_BAND=<m-tiles per band of the tile sweep>
+ * override the choice; they are read on every call. */
 sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A,
                       const void* meta, const void* B, const void* beta, const void* C,
                       void* D, void* workspace, size_t workspace_bytes, void* stream);

@@ -55,6 +55,8 @@ struct GemmParams {
   int32_t cd_type;    // sp24_dtype of C / D
   int32_t has_c;
   int32_t stages, epi_bytes;  // shared memory: ring stages and bytes of epilogue staging
+  long long wait_limit;       // SM cycles after which a device-side wait gives up
+  int32_t test_skip_stage;    // test hook: the producers leave out one k-block, so that a wait expires
   int32_t band;       // m-tiles per band of the tile sweep
   int32_t cd_col_major;  // C and D stored M-contiguous (the [tokens, out_features] layout)
   // implicit 3x3 convolution: B is the im2col view of an NHWC activation (never materialised)
@@ -117,7 +119,7 @@ struct Shared {
 static_assert(sizeof(Shared) <= 512, "barrier block");
 
 __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, Shared* sh, uint32_t* status,
-                                             uint32_t code) {
+                                             uint32_t code, long long limit) {
   // fast path: poll a while before any bookkeeping; try_wait itself suspends the thread briefly
 #pragma unroll 1
   for (int i = 0; i < 64; ++i)
@@ -128,7 +130,7 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, Sha
     if (ptx::mbar_try_wait(bar, parity)) return true;
     if ((++spins & 255u) == 0) {
       if (sh->abort) return false;
-      if (clock64() - t0 > kWaitTimeoutCycles) {
+      if (clock64() - t0 > limit) {
         sh->abort = 1;
         atomicCAS(status, 0u, code);
         return false;
@@ -418,7 +420,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           conv_q = rem - conv_p * p.conv_w;
         }
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!bounded_wait(&sh->empty[stage], phase ^ 1u, sh, p.status, 1u)) break;
+          if (!bounded_wait(&sh->empty[stage], phase ^ 1u, sh, p.status, 1u, p.wait_limit)) break;
+          if (p.test_skip_stage && t == cluster_id && kb == 1) {
+            // test hook: this k-block of the first tile is neither armed nor loaded by either CTA, so
+            // the MMA issuer's wait for it expires and every role leaves through the abort path
+            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           uint8_t* sa = smem + stage * C::kStageBytes;
           uint8_t* sb = sa + C::kABytes;
           uint8_t* se = sb + C::kBBytes;
@@ -490,11 +498,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int live = min(MBLK, (int)((p.M - (int64_t)mt * MBLK * CTAS * kBlockM + CTAS * kBlockM - 1) /
                                          (CTAS * kBlockM)));
         const uint32_t idesc = make_idesc<KIND>(SPARSE, B_MN, p.a_fmt, kBlockM * CTAS, n_eff);
-        if (!bounded_wait(&sh->tmem_empty[acc], acc_phase ^ 1u, sh, p.status, 2u)) break;
+        if (!bounded_wait(&sh->tmem_empty[acc], acc_phase ^ 1u, sh, p.status, 2u, p.wait_limit)) break;
         ptx::tc_fence_after();
         bool ok = true;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!bounded_wait(&sh->full[stage], phase, sh, p.status, 3u)) { ok = false; break; }
+          if (!bounded_wait(&sh->full[stage], phase, sh, p.status, 3u, p.wait_limit)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sa = ptx::smem_u32(smem + stage * C::kStageBytes);
           const uint32_t sb = sa + C::kABytes;
@@ -615,7 +623,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
       int mt, nt;
       tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
-      if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u)) break;
+      if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u, p.wait_limit)) break;
       ptx::tc_fence_after();
       uint32_t r_next[32];
       const uint32_t t_acc = tmem_base + (acc * MBLK) * BLOCK_N + ((uint32_t)(q * 32) << 16);
@@ -638,7 +646,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (!box_of(mt, nt, it, row0, col0)) continue;  // same answer for the whole warp
         const int b = seq % nbuf;
         uint8_t* buf = my_bufs + b * buf_bytes;
-        if (p.has_c && !bounded_wait(&sh->c_full[ew][b], (seq / nbuf) & 1u, sh, p.status, 5u)) { ok = false; break; }
+        if (p.has_c && !bounded_wait(&sh->c_full[ew][b], (seq / nbuf) & 1u, sh, p.status, 5u, p.wait_limit)) { ok = false; break; }
         if (KIND == 1 && p.dequant) {
           // this thread's output row: its scale and bias
           const int row = min(row0 + lane, (int)p.M - 1);
@@ -979,6 +987,14 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   p.a_fmt = (d->ab_type == SP24_BF16 || d->ab_type == SP24_E5M2) ? 1 : 0;
   p.cd_type = (int)d->cd_type;
   p.has_c = has_c ? 1 : 0;
+  p.wait_limit = kWaitTimeoutCycles;
+  // Test hooks for the failure path (tests/test_gpu_timeout.py): a shorter limit, and a pipeline that
+  // stalls by leaving out one k-block.  Nothing faults or hangs: the waits expire and the kernel returns.
+  if (const char* env = getenv("SP24_TEST_WAIT_CYCLES")) {
+    const long long v = atoll(env);
+    if (v >= 1000000) p.wait_limit = v;
+  }
+  if (const char* env = getenv("SP24_TEST_SKIP_STAGE")) p.test_skip_stage = atoi(env) != 0;
   p.cd_col_major = d->order_d == SP24_COL_MAJOR ? 1 : 0;
   const bool sparse = !d->a_is_dense;
   const bool i8 = d->ab_type == SP24_I8, tf32 = d->ab_type == SP24_F32, f8 = is_fp8(d->ab_type);

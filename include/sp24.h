@@ -191,7 +191,8 @@ size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d);
  * The tile shape is chosen from the problem size.  For benchmarking the environment variables
  * SP24_TILE=<CTAs per tile: 1|2>x<columns per tile>x<128-row blocks per CTA: 1|2> (one of the
  * built shapes, else SP24_ERR_UNSUPPORTED) and SP24_BAND=<m-tiles per band of the tile sweep>
- * override the choice; they are read on every call. */
+ * override the choice; they are read on every call.  SP24_LOG=1 prints the problem and the chosen
+ * tile shape of every call to stderr. */
 sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A,
                       const void* meta, const void* B, const void* beta, const void* C,
                       void* D, void* workspace, size_t workspace_bytes, void* stream);

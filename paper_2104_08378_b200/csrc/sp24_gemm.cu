@@ -1024,6 +1024,11 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
     if (b > 0) p.band = b;
   }
   const bool b_mn = d->order_b == SP24_ROW_MAJOR;  // B stored N-contiguous
+  if (getenv("SP24_LOG"))
+    fprintf(stderr, "sp24_gemm: M=%lld N=%lld K=%lld ab=%d cd=%d %s%s tile=%dx%dx%d band=%d beta=%g%s%s\n", (long long)d->M,
+            (long long)d->N, (long long)d->K, (int)d->ab_type, (int)d->cd_type, sparse ? "sparse" : "dense",
+            b_mn ? " B:N-contiguous" : "", ctas, block_n, mblk, p.band, (double)fbeta, dq ? " dequant" : "",
+            cv ? " conv3x3" : "");
 #define SP24_LAUNCH(K_, BN, CT, MB, MN)                                                               \
   (sparse ? launch<K_, true, BN, CT, MB, MN>(d, p, A, meta, B, s) : launch<K_, false, BN, CT, MB, MN>(d, p, A, meta, B, s))
 #define SP24_DISPATCH(CT, BN, MB)                                                                     \

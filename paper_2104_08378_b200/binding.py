@@ -174,12 +174,13 @@ def prune_compress(x: torch.Tensor, layout: int = META_TCGEN05, dtype: str | Non
 
 
 def decompress(vals: torch.Tensor, meta: torch.Tensor, layout: int = META_TCGEN05,
-               dtype: str | None = None) -> torch.Tensor:
+               dtype: str | None = None, out: torch.Tensor | None = None) -> torch.Tensor:
     dt = _dtype_of(vals, dtype)
     M, K2 = vals.shape
-    y = torch.empty((M, 2 * K2), dtype=vals.dtype, device=vals.device)
+    y = torch.empty((M, 2 * K2), dtype=vals.dtype, device=vals.device) if out is None else out
     _check(lib.sp24_decompress(DTYPE_CODE[dt], M, 2 * K2, _ptr(vals), vals.stride(0) if M > 1 else K2,
-                               _ptr(meta), layout, _ptr(y), 2 * K2, _stream()), "sp24_decompress")
+                               _ptr(meta), layout, _ptr(y), y.stride(0) if M > 1 else 2 * K2, _stream()),
+           "sp24_decompress")
     return y
 
 
@@ -234,11 +235,12 @@ def gemm_status(ws: torch.Tensor | None = None, device=None) -> int:
     return lib.sp24_gemm_status(_ptr(ws), _stream())
 
 
-def im2col_nhwc_3x3(x: torch.Tensor, dtype: str | None = None) -> torch.Tensor:
+def im2col_nhwc_3x3(x: torch.Tensor, dtype: str | None = None, out: torch.Tensor | None = None) -> torch.Tensor:
     dt = _dtype_of(x, dtype)
     Nb, H, W, C = x.shape
-    out = torch.empty((Nb * H * W, 9 * C), dtype=x.dtype, device=x.device)
-    _check(lib.sp24_im2col_nhwc_3x3(DTYPE_CODE[dt], Nb, H, W, C, _ptr(x), _ptr(out), 9 * C, _stream()),
+    if out is None:
+        out = torch.empty((Nb * H * W, 9 * C), dtype=x.dtype, device=x.device)
+    _check(lib.sp24_im2col_nhwc_3x3(DTYPE_CODE[dt], Nb, H, W, C, _ptr(x), _ptr(out), out.stride(0), _stream()),
            "sp24_im2col_nhwc_3x3")
     return out
 

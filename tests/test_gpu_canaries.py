@@ -57,6 +57,10 @@ def test_streaming_kernels_stay_inside_their_outputs(sp, dtype, shape):
             torch.cuda.synchronize()
             vals.check("compress values")
             meta.check("compress metadata")
+            back = Guarded(M, K, dtype, K + ld_extra)
+            sp.decompress(vals.t, meta.t.view(-1), layout=layout, out=back.t)
+            torch.cuda.synchronize()
+            back.check("decompress")
             if name != "f32":
                 p2, v2, m2 = Guarded(M, K, dtype, K + ld_extra), Guarded(M, K // 2, dtype), Guarded(1, meta.cols, torch.uint8)
                 sp.prune_compress(x, layout=layout, pruned=p2.t, vals=v2.t, meta=m2.t.view(-1))
@@ -93,3 +97,16 @@ def test_gemm_stays_inside_d(sp, monkeypatch, kind, tile):
         sp.gemm(vals, meta, Bt, out=Dt.t, cd=cd, cd_col_major=True, ws=ws)
         torch.cuda.synchronize()
         Dt.check(f"gemm {kind} {tile} column-major")
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.int8])
+@pytest.mark.parametrize("shape", [(3, 5, 7, 64), (2, 14, 14, 256), (1, 1, 1, 16)])
+def test_im2col_stays_inside_its_output(sp, dtype, shape):
+    Nb, H, W, C = shape
+    x = torch.randint(-100, 100, shape, device="cuda").to(dtype)
+    for ld_extra in (0, 16):
+        out = Guarded(Nb * H * W, 9 * C, dtype, 9 * C + ld_extra)
+        sp.im2col_nhwc_3x3(x, out=out.t)
+        torch.cuda.synchronize()
+        out.check("im2col")
+        assert torch.equal(out.t.contiguous(), sp.im2col_nhwc_3x3(x))

@@ -60,12 +60,17 @@ def _run_config(sp, cfg, Bt, full_gemm):
     # prune, compress, metadata: bit-exact, in full
     pruned = sp.prune(Ad)
     vals, meta, dropped = sp.compress(pruned, layout=sp.META_TCGEN05, count_dropped=True)
-    vals_ref, meta_ref, _ = oracle.compress(A, ab)
+    vals_ref, meta_ref, dropped_ref = oracle.compress(A, ab)
     assert np.array_equal(to_host_bits(pruned), oracle.prune(A, ab))
     assert np.array_equal(to_host_bits(vals), vals_ref)
     assert np.array_equal(meta.cpu().numpy(), oracle.meta_to_operand_order(meta_ref, ab))
     assert int(dropped.item()) == 0
-    del Ad
+    # the same three outputs from the one-pass entry point (what the benchmark's step launches)
+    pruned_f, vals_f, meta_f, dropped_f = sp.prune_compress(Ad, layout=sp.META_TCGEN05, count_dropped=True)
+    assert torch.equal(pruned_f.view(torch.uint8), pruned.view(torch.uint8))
+    assert torch.equal(vals_f.view(torch.uint8), vals.view(torch.uint8)) and torch.equal(meta_f, meta)
+    assert int(dropped_f.item()) == dropped_ref
+    del Ad, pruned_f, vals_f, meta_f
     for dense in (False, True):
         if dense:
             D = sp.gemm(pruned, None, Btd, alpha=cfg.alpha, beta=cfg.beta, C=Cd, cd=cd, a_is_dense=True)

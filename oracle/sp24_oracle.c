@@ -19,7 +19,8 @@
  * C(4,2) keep-patterns, the metadata example of Section 3.1, the storage arithmetic of
  * Section 3.1, decompress(compress(x)) == prune(x), sparse GEMM == library dense matmul on
  * the pruned matrix, closed forms (identity B, all-ones), a direct 7-loop convolution for
- * im2col, and hand-computed positions for the tensor-core metadata permutation.
+ * im2col, hand-computed positions for the tensor-core metadata permutation, and for the
+ * error-bound scale (|A| . |B|) a library matmul of the magnitudes plus its closed forms.
  */
 #include <math.h>
 #include <stdint.h>

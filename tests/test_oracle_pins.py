@@ -220,6 +220,35 @@ def test_sparse_gemm_equals_library_matmul_on_pruned_matrix(dtype):
     assert np.array_equal(sub, D[5:9, 3:17])
 
 
+@pytest.mark.parametrize("dtype", ["f16", "bf16", "e4m3", "e5m2"])
+def test_gemm_abs_equals_library_matmul_of_magnitudes(dtype):
+    """The scale of the per-element error bound, (|A| . |B|)_ij over the kept values: equal to a
+    numpy float64 matmul of the magnitudes of the decompressed matrix and of B, in full and on a
+    window (an inflated scale -- a sum over the wrong range, a wrong leading dimension -- would
+    loosen every floating-point parity test without failing any of them)."""
+    M, N, K = 28, 36, 96
+    x = _rand(dtype, M, K, 61)
+    x[::3, 1::4] = 0                                   # some groups with fillers (zeros that are stored)
+    Bt = _rand(dtype, N, K, 62, ("uniform", -1.0, 1.0))
+    vals, meta, _ = oracle.compress(x, dtype)
+    lib = np.abs(_f64(oracle.decompress(vals, meta, dtype), dtype)) @ np.abs(_f64(Bt, dtype)).T
+    got = oracle.gemm_abs(vals, meta, Bt, dtype)
+    assert got.shape == (M, N) and np.all(got >= 0)
+    assert np.all(np.abs(got - lib) <= 1e-13 * lib + 1e-300)
+    sub = oracle.gemm_abs(vals, meta, Bt, dtype, rows=(4, 13), cols=(7, 30))
+    assert np.array_equal(sub, got[4:13, 7:30])
+    # it bounds the signed product, and meets it when every term has one sign
+    D = oracle.gemm_sparse(vals, meta, Bt, dtype)
+    assert np.all(np.abs(D) <= got * (1 + 1e-13))
+    pos_a, pos_b = x & (0x7F if dtype in ("e4m3", "e5m2") else 0x7FFF), Bt & (0x7F if dtype in ("e4m3", "e5m2") else 0x7FFF)
+    vp, mp, _ = oracle.compress(pos_a, dtype)
+    assert np.array_equal(oracle.gemm_abs(vp, mp, pos_b, dtype), oracle.gemm_sparse(vp, mp, pos_b, dtype))
+    # all ones: K/2 kept products of 1 each
+    ones_a, ones_b = _from_float(np.ones((4, K)), dtype), _from_float(-np.ones((6, K)), dtype)
+    v1, m1, _ = oracle.compress(ones_a, dtype)
+    assert np.all(oracle.gemm_abs(v1, m1, ones_b, dtype) == K // 2)
+
+
 @pytest.mark.parametrize("dtype", DTYPES)
 def test_gemm_closed_forms(dtype):
     K = 32

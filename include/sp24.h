@@ -184,15 +184,13 @@ size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d);
  *   A:    device; vals (M x K/2) or dense A (M x K), row-major, 16-byte aligned.
  *   meta: device; TCGEN05-layout metadata of A (ignored when a_is_dense).
  *   B, C, D: device, 16-byte aligned.  C may be NULL iff beta == 0.  C may alias D.
- *   workspace: device, >= sp24_gemm_workspace_bytes(d).  The kernel writes a status record
- *              there; read it back with sp24_gemm_status after synchronising.
+ *   workspace: device, >= sp24_gemm_workspace_bytes(d), zero-filled before its first use.  The
+ *              kernel records an expired wait there; see sp24_gemm_status.
  * Accumulation is FP32 (INT32) in hardware order; the result is rounded to cd_type once,
  * round-to-nearest-even.
- * The tile shape is chosen from the problem size.  For benchmarking the environment variables
- * SP24_TILE=<CTAs per tile: 1|2>x<columns per tile>x<128-row blocks per CTA: 1|2> (one of the
- * built shapes, else SP24_ERR_UNSUPPORTED) and SP24_BAND=<m-tiles per band of the tile sweep>
- * override the choice; they are read on every call.  SP24_LOG=1 prints the problem and the chosen
- * tile shape of every call to stderr. */
+ * The tile shape is chosen from the problem size (sp24_set_tile_override forces one).
+ * The five tensor maps of a call are kept in a small per-thread host cache keyed by address,
+ * shape and leading dimension, so repeated calls on the same buffers do not encode them again. */
 sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A,
                       const void* meta, const void* B, const void* beta, const void* C,
                       void* D, void* workspace, size_t workspace_bytes, void* stream);
@@ -230,10 +228,16 @@ sp24_status sp24_conv3x3_nhwc(const sp24_gemm_desc* d, int64_t Nb, int64_t H, in
                               const void* beta, const void* C, void* D, void* workspace,
                               size_t workspace_bytes, void* stream);
 
-/* Copies the status record of the last sp24_gemm that used `workspace` back to the host
- * (synchronises `stream`) and returns SP24_OK, or SP24_ERR_TIMEOUT if a bounded wait inside
- * the kernel expired (the kernel then returned early and D is incomplete). */
-sp24_status sp24_gemm_status(const void* workspace, void* stream);
+/* Reads the status record in `workspace` back to the host (synchronises `stream`) and returns
+ * SP24_OK, or SP24_ERR_TIMEOUT if a bounded wait inside any GEMM kernel that used this workspace
+ * since the last read expired (that kernel returned early and its D is incomplete).
+ * The record is STICKY: `workspace` must be zero-filled once before its first use (e.g.
+ * cudaMemsetAsync); the kernels never clear it, they only write the code of the first wait that
+ * expired into word 0 and count expired waits in word 1.  One record therefore covers any number
+ * of launches (a benchmark loop, the bands of sp24_pipeline_host): a timeout in any of them is
+ * still there when this call reads it.  A reported timeout is cleared by this call (a memset on
+ * `stream`), so that the next read concerns the launches that follow. */
+sp24_status sp24_gemm_status(void* workspace, void* stream);
 
 /* (No counterpart in the paper: a deployment variant of sp24_gemm.)
  * sp24_gemm for callers that cannot allocate device memory -- a process whose framework
@@ -245,12 +249,36 @@ sp24_status sp24_gemm_status(const void* workspace, void* stream);
  * results are those of sp24_gemm; inputs and outputs remain the caller's buffers.
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress);
  * make that first call before any stream capture.  Nothing is allocated or freed.
- * All calls on a device share the array and its status word is cleared on the stream before
- * each launch, so two calls that overlap on the GPU (different streams) race: serialise them.
- * The status record of this variant cannot be read back with sp24_gemm_status. */
+ * All calls on a device share the array.  It starts zero-filled and nothing has to be cleared
+ * between calls: the kernels only write into it when a bounded wait expires, and the record
+ * then stays until sp24_gemm_static_ws_status reads it.  Two calls that overlap on the GPU
+ * (different streams) share the one record, so a timeout cannot be attributed to one of them:
+ * serialise such calls, or use sp24_gemm with a workspace per stream. */
 sp24_status sp24_gemm_static_ws(const sp24_gemm_desc* d, const void* alpha, const void* A,
                                 const void* meta, const void* B, const void* beta,
                                 const void* C, void* D, void* stream);
+
+/* (No counterpart in the paper.)  sp24_gemm_status for the array of sp24_gemm_static_ws on the
+ * current device: synchronises `stream`, returns SP24_OK or SP24_ERR_TIMEOUT (and then clears
+ * the record).  Allocates nothing. */
+sp24_status sp24_gemm_static_ws_status(void* stream);
+
+/* Benchmarking and test support (no counterpart in the paper): forces the tile shape of every
+ * following sp24_gemm / sp24_gemm_i8_dequant / sp24_conv3x3_nhwc call in this process.
+ *   ctas: 1 or 2 CTAs per tile; block_n: columns per tile; mblk: 128-row blocks per CTA (1 or 2);
+ *   the shape must be one of the built ones, else those calls return SP24_ERR_UNSUPPORTED.
+ *   ctas == 0 restores the automatic choice.  band: m-tiles per band of the tile sweep, 0 = default.
+ * The environment variables SP24_TILE=<ctas>x<block_n>x<mblk>, SP24_BAND=<band> and SP24_LOG=1
+ * (print the problem and the chosen tile shape of every call to stderr) give the initial values;
+ * they are read ONCE, at the first GEMM call of the process. */
+sp24_status sp24_set_tile_override(int ctas, int block_n, int mblk, int band);
+
+/* Test support for the failure path, not for production use: shortens the limit of every
+ * device-side wait to `wait_cycles` SM cycles (values below 1 000 000 restore the default of
+ * about a second) and, with skip_stage != 0, makes the TMA producers leave out one k-block of
+ * their first tile so that a wait expires.  Nothing faults or hangs: the kernel returns early
+ * and sp24_gemm_status reports SP24_ERR_TIMEOUT.  Never read from the environment. */
+sp24_status sp24_test_set_fault_hooks(long long wait_cycles, int skip_stage);
 
 /* Lowering of a 3x3, stride-1, pad-1 NHWC convolution input to the GEMM's B operand
  * (Section 4.2: a convolution's reduction dimension is C*R*S).  Output is K-contiguous:
@@ -297,7 +325,8 @@ sp24_status sp24_prune_2d(sp24_dtype t, int64_t M, int64_t K, const void* x, int
  * in up to eight row bands: each band's D is copied out on a second, library-owned stream
  * (created once per device; `stream` is made to wait for it before the call returns) while
  * the next band's A and C are copied in, so both directions of the host link are busy.  The status
- * word in `workspace` then reflects the last band only. */
+ * record in `workspace` is sticky (see sp24_gemm_status), so it covers every band.  The call may be
+ * made from several host threads at once (events are created per call). */
 sp24_status sp24_pipeline_host(const sp24_gemm_desc* d, const void* alpha, const void* h_A,
                                const void* h_B, const void* beta, const void* h_C, void* h_D,
                                void* d_A, void* d_vals, void* d_meta, void* d_B, void* d_C,

@@ -32,6 +32,7 @@ EXPORTS = [
     "sp24_decompress", "sp24_prune_compress", "sp24_gemm_workspace_bytes", "sp24_gemm", "sp24_gemm_status",
     "sp24_im2col_nhwc_3x3", "sp24_pipeline_host", "sp24_gemm_static_ws", "sp24_gemm_i8_dequant",
     "sp24_conv3x3_nhwc", "sp24_kept_magnitude", "sp24_apply_mask", "sp24_prune_2d",
+    "sp24_gemm_static_ws_status", "sp24_set_tile_override", "sp24_test_set_fault_hooks",
 ]
 
 
@@ -82,6 +83,12 @@ def _load() -> ctypes.CDLL:
     for name in ("sp24_kept_magnitude", "sp24_apply_mask", "sp24_prune_2d"):
         getattr(lib, name).restype = ci
     lib.sp24_gemm_status.argtypes = [vp, vp]
+    lib.sp24_gemm_static_ws_status.argtypes = [vp]
+    lib.sp24_gemm_static_ws_status.restype = ci
+    lib.sp24_set_tile_override.argtypes = [ci, ci, ci, ci]
+    lib.sp24_set_tile_override.restype = ci
+    lib.sp24_test_set_fault_hooks.argtypes = [ctypes.c_longlong, ci]
+    lib.sp24_test_set_fault_hooks.restype = ci
     lib.sp24_im2col_nhwc_3x3.argtypes = [ci, i64, i64, i64, i64, vp, vp, i64, vp]
     lib.sp24_pipeline_host.argtypes = [ctypes.POINTER(GemmDesc)] + [vp] * 13 + [sz, vp]
     for name in ("sp24_prune", "sp24_compress", "sp24_decompress", "sp24_gemm", "sp24_gemm_status",
@@ -231,8 +238,27 @@ def gemm(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor, *, alpha=
 
 
 def gemm_status(ws: torch.Tensor | None = None, device=None) -> int:
+    """sp24_gemm_status: 0, or SP24_ERR_TIMEOUT (9) if a wait expired in any launch on this workspace
+    since the last read (the record is then cleared)."""
     ws = ws if ws is not None else workspace(device or "cuda")
     return lib.sp24_gemm_status(_ptr(ws), _stream())
+
+
+def gemm_static_ws_status() -> int:
+    """sp24_gemm_static_ws_status: the same for the library's own workspace array on the current device."""
+    return lib.sp24_gemm_static_ws_status(_stream())
+
+
+def set_tile_override(tile: str | None = None, band: int = 0):
+    """sp24_set_tile_override: tile = "<ctas>x<block_n>x<mblk>" forces that tile shape, None restores
+    the automatic choice (benchmarks and tests)."""
+    c, n, m = (0, 0, 0) if not tile else (list(map(int, tile.split("x"))) + [1])[:3]
+    _check(lib.sp24_set_tile_override(c, n, m, band), "sp24_set_tile_override")
+
+
+def set_fault_hooks(wait_cycles: int = 0, skip_stage: bool = False):
+    """sp24_test_set_fault_hooks (failure-path tests only)."""
+    _check(lib.sp24_test_set_fault_hooks(int(wait_cycles), 1 if skip_stage else 0), "sp24_test_set_fault_hooks")
 
 
 def im2col_nhwc_3x3(x: torch.Tensor, dtype: str | None = None, out: torch.Tensor | None = None) -> torch.Tensor:

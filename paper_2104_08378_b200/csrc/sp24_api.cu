@@ -64,32 +64,41 @@ extern "C" size_t sp24_meta_bytes(sp24_dtype t, int64_t M, int64_t K, sp24_meta_
 
 namespace {
 
-// Second stream and events of the host-buffer pipeline, created once per device and kept.
+// Second stream of the host-buffer pipeline, created once per device and kept (a stream holds no
+// device memory).  It is shared by all callers; what orders one call's copies behind its own
+// GEMMs are events, and those are created per call (see BandEvents), so calls from several host
+// threads do not disturb one another.
 constexpr int kMaxBands = 8;
-struct SideStream {
-  cudaStream_t stream = nullptr;
-  cudaEvent_t band_done[kMaxBands] = {};
-  cudaEvent_t joined = nullptr;
-  bool ready = false;
-};
 
-sp24_status side_stream(SideStream** out) {
+sp24_status side_stream(cudaStream_t* out) {
   static std::mutex mu;
-  static SideStream per_device[64];
+  static cudaStream_t per_device[64] = {};
   int dev = 0;
   SP24_CUDA_CHECK(cudaGetDevice(&dev));
   SP24_RETURN_IF(dev < 0 || dev >= 64, SP24_ERR_UNSUPPORTED);
   std::lock_guard<std::mutex> lock(mu);
-  SideStream& ss = per_device[dev];
-  if (!ss.ready) {
-    SP24_CUDA_CHECK(cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking));
-    for (int b = 0; b < kMaxBands; ++b) SP24_CUDA_CHECK(cudaEventCreateWithFlags(&ss.band_done[b], cudaEventDisableTiming));
-    SP24_CUDA_CHECK(cudaEventCreateWithFlags(&ss.joined, cudaEventDisableTiming));
-    ss.ready = true;
-  }
-  *out = &ss;
+  if (per_device[dev] == nullptr) SP24_CUDA_CHECK(cudaStreamCreateWithFlags(&per_device[dev], cudaStreamNonBlocking));
+  *out = per_device[dev];
   return SP24_OK;
 }
+
+// The events of ONE sp24_pipeline_host call: one per band (GEMM done -> copy-out may start) and
+// one for the final join.  Destroyed when the call returns; an event that is still pending is
+// released by the runtime once it has completed.
+struct BandEvents {
+  cudaEvent_t band_done[kMaxBands] = {};
+  cudaEvent_t joined = nullptr;
+  sp24_status create(int bands) {
+    for (int b = 0; b < bands; ++b) SP24_CUDA_CHECK(cudaEventCreateWithFlags(&band_done[b], cudaEventDisableTiming));
+    SP24_CUDA_CHECK(cudaEventCreateWithFlags(&joined, cudaEventDisableTiming));
+    return SP24_OK;
+  }
+  ~BandEvents() {
+    for (cudaEvent_t e : band_done)
+      if (e) cudaEventDestroy(e);
+    if (joined) cudaEventDestroy(joined);
+  }
+};
 
 }  // namespace
 
@@ -118,22 +127,28 @@ extern "C" sp24_status sp24_pipeline_host(const sp24_gemm_desc* d, const void* a
   int bands = (int)(d->M / 8192);
   bands = bands < 1 ? 1 : (bands > kMaxBands ? kMaxBands : bands);
   const int64_t band_rows = bands == 1 ? d->M : ((d->M + bands - 1) / bands + 511) / 512 * 512;
-  SideStream* ss = nullptr;
-  if (bands > 1 && (st = side_stream(&ss)) != SP24_OK) return st;
+  cudaStream_t side = nullptr;
+  BandEvents ev;
+  if (bands > 1) {
+    if ((st = side_stream(&side)) != SP24_OK) return st;
+    if ((st = ev.create(bands)) != SP24_OK) return st;
+  }
   const size_t meta_block_bytes = sp24_meta_bytes(d->ab_type, 128, d->K, SP24_META_TCGEN05);  // per 128 rows
   int issued = 0;
-  for (int b = 0; b < bands; ++b) {
+  // one band; any failure leaves through the join below, so that copies already queued on the
+  // second stream are ordered before whatever the caller enqueues next
+  auto run_band = [&](int b) -> sp24_status {
     const int64_t r0 = (int64_t)b * band_rows, r1 = r0 + band_rows < d->M ? r0 + band_rows : d->M;
-    if (r0 >= r1) break;
+    if (r0 >= r1) return SP24_OK;
     const size_t c_off = (size_t)r0 * d->N * cs, c_bytes = (size_t)(r1 - r0) * d->N * cs;
     const size_t a_off = (size_t)r0 * d->K * es, v_off = (size_t)r0 * (d->K / 2) * es;
     const size_t m_off = (size_t)(r0 / 128) * meta_block_bytes;
     SP24_CUDA_CHECK(cudaMemcpyAsync(static_cast<char*>(d_A) + a_off, static_cast<const char*>(h_A) + a_off,
                                     (size_t)(r1 - r0) * d->K * es, cudaMemcpyHostToDevice, s));
-    st = sp24_compress(d->ab_type, r1 - r0, d->K, static_cast<const char*>(d_A) + a_off, d->K,
-                       static_cast<char*>(d_vals) + v_off, d->K / 2, static_cast<char*>(d_meta) + m_off,
-                       SP24_META_TCGEN05, nullptr, stream);
-    if (st != SP24_OK) break;
+    sp24_status bs = sp24_compress(d->ab_type, r1 - r0, d->K, static_cast<const char*>(d_A) + a_off, d->K,
+                                   static_cast<char*>(d_vals) + v_off, d->K / 2, static_cast<char*>(d_meta) + m_off,
+                                   SP24_META_TCGEN05, nullptr, stream);
+    if (bs != SP24_OK) return bs;
     if (has_c)
       SP24_CUDA_CHECK(cudaMemcpyAsync(static_cast<char*>(d_C) + c_off, static_cast<const char*>(h_C) + c_off, c_bytes,
                                       cudaMemcpyHostToDevice, s));
@@ -143,24 +158,28 @@ extern "C" sp24_status sp24_pipeline_host(const sp24_gemm_desc* d, const void* a
     packed.ldb = d->K;
     packed.ldc = d->N;
     packed.ldd = d->N;
-    st = sp24_gemm(&packed, alpha, static_cast<const char*>(d_vals) + v_off,
-                   static_cast<const char*>(d_meta) + m_off, d_B, beta,
-                   has_c ? static_cast<const char*>(d_C) + c_off : nullptr, static_cast<char*>(d_D) + c_off, workspace,
-                   workspace_bytes, stream);
-    if (st != SP24_OK) break;
+    bs = sp24_gemm(&packed, alpha, static_cast<const char*>(d_vals) + v_off, static_cast<const char*>(d_meta) + m_off,
+                   d_B, beta, has_c ? static_cast<const char*>(d_C) + c_off : nullptr, static_cast<char*>(d_D) + c_off,
+                   workspace, workspace_bytes, stream);
+    if (bs != SP24_OK) return bs;
     cudaStream_t out = s;
     if (bands > 1) {
-      SP24_CUDA_CHECK(cudaEventRecord(ss->band_done[b], s));
-      SP24_CUDA_CHECK(cudaStreamWaitEvent(ss->stream, ss->band_done[b], 0));
-      out = ss->stream;
+      SP24_CUDA_CHECK(cudaEventRecord(ev.band_done[b], s));
+      SP24_CUDA_CHECK(cudaStreamWaitEvent(side, ev.band_done[b], 0));
+      out = side;
       ++issued;
     }
     SP24_CUDA_CHECK(cudaMemcpyAsync(static_cast<char*>(h_D) + c_off, static_cast<const char*>(d_D) + c_off, c_bytes,
                                     cudaMemcpyDeviceToHost, out));
-  }
-  if (issued) {  // the caller's stream ends behind every copy made on the second one
-    SP24_CUDA_CHECK(cudaEventRecord(ss->joined, ss->stream));
-    SP24_CUDA_CHECK(cudaStreamWaitEvent(s, ss->joined, 0));
+    return SP24_OK;
+  };
+  for (int b = 0; b < bands && st == SP24_OK; ++b) st = run_band(b);
+  if (issued) {  // the caller's stream ends behind every copy made on the second one, also after a failure
+    const bool joined = cudaEventRecord(ev.joined, side) == cudaSuccess && cudaStreamWaitEvent(s, ev.joined, 0) == cudaSuccess;
+    if (!joined) {
+      cudaStreamSynchronize(side);  // last resort: order by waiting on the host
+      if (st == SP24_OK) st = SP24_ERR_CUDA;
+    }
   }
   return st;
 }

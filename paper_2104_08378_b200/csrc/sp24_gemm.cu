@@ -19,12 +19,14 @@
 // two m-blocks cuts the bytes per flop by about a third.  The two accumulators then fill tensor
 // memory, so the epilogue is not overlapped with the next tile's main loop; MBLK == 1 keeps two
 // accumulator buffers and overlaps it.
-// Every wait is bounded: on expiry the role records a code in the status word and all roles
-// leave through the normal teardown (no trap, no endless spin).
+// Every wait is bounded: on expiry the role records a code in the status record and all roles
+// leave through the normal teardown (no trap, no endless spin).  The kernel never clears the
+// record: it stays at the first expired wait, across launches, until the host reads it.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 #include <mutex>
@@ -47,7 +49,7 @@ struct GemmParams {
   int64_t ldc, ldd;   // elements
   const void* C;
   void* D;
-  uint32_t* status;   // [0] = 0 ok, else code of the wait that expired
+  uint32_t* status;   // [0] = 0 ok, else code of the first wait that expired; [1] = number of expired waits
   float alpha, beta;
   int32_t m_tiles, n_tiles, k_blocks;
   int32_t meta_kb;    // 128-column metadata blocks per 128-row block (K padded to 256)
@@ -132,7 +134,8 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, Sha
       if (sh->abort) return false;
       if (clock64() - t0 > limit) {
         sh->abort = 1;
-        atomicCAS(status, 0u, code);
+        atomicCAS(status, 0u, code);   // sticky: the first code stays until the host reads and clears it
+        atomicAdd(status + 1, 1u);
         return false;
       }
     }
@@ -377,7 +380,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     for (int w = 0; w < kEpiWarps; ++w)
       for (int b = 0; b < 4; ++b) ptx::mbar_init(&sh->c_full[w][b], 1);
     sh->abort = 0;
-    if (blockIdx.x == 0) p.status[0] = 0;  // a wait can only expire a second later
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&map_a);
     ptx::prefetch_tensormap(&map_b);
@@ -759,8 +761,8 @@ sp24_status make_im2col_map(CUtensorMap* map, const void* x, int es, uint64_t nb
 
 // 2-D tensor map over a row-major (rows x cols) array of `es`-byte elements with `ld_bytes`
 // between rows; box = box_cols x box_rows elements.
-sp24_status make_map(CUtensorMap* map, const void* base, int es, uint64_t rows, uint64_t cols, uint64_t ld_bytes,
-                     uint32_t box_cols, uint32_t box_rows, int swizzle_bytes) {
+sp24_status encode_map(CUtensorMap* map, const void* base, int es, uint64_t rows, uint64_t cols, uint64_t ld_bytes,
+                       uint32_t box_cols, uint32_t box_rows, int swizzle_bytes) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return SP24_ERR_CUDA;
   cuuint64_t dims[2] = {cols, rows};
@@ -776,14 +778,74 @@ sp24_status make_map(CUtensorMap* map, const void* base, int es, uint64_t rows, 
   return r == CUDA_SUCCESS ? SP24_OK : SP24_ERR_CUDA;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+// Host-side cache of encoded tensor maps.  A map is a pure function of (address, shape, leading
+// dimension, element size, box, swizzle): a layer that is multiplied again with the same buffers
+// finds its five maps here instead of encoding them again.  One small table per host thread (no
+// lock), replaced round-robin.
+struct MapKey {
+  const void* base;
+  uint64_t rows, cols, ld_bytes;
+  uint32_t box_cols, box_rows;
+  int32_t es, swizzle;
+  bool operator==(const MapKey& o) const {
+    return base == o.base && rows == o.rows && cols == o.cols && ld_bytes == o.ld_bytes && box_cols == o.box_cols &&
+           box_rows == o.box_rows && es == o.es && swizzle == o.swizzle;
   }
+};
+struct MapCache {
+  static constexpr int kEntries = 32;
+  MapKey keys[kEntries];
+  CUtensorMap maps[kEntries];
+  int used = 0, next = 0;
+};
+
+sp24_status make_map(CUtensorMap* map, const void* base, int es, uint64_t rows, uint64_t cols, uint64_t ld_bytes,
+                     uint32_t box_cols, uint32_t box_rows, int swizzle_bytes) {
+  static thread_local MapCache cache;
+  const MapKey key = {base, rows, cols, ld_bytes, box_cols, box_rows, es, swizzle_bytes};
+  for (int i = 0; i < cache.used; ++i)
+    if (cache.keys[i] == key) {
+      *map = cache.maps[i];
+      return SP24_OK;
+    }
+  sp24_status st = encode_map(map, base, es, rows, cols, ld_bytes, box_cols, box_rows, swizzle_bytes);
+  if (st != SP24_OK) return st;
+  const int slot = cache.used < MapCache::kEntries ? cache.used++ : (cache.next++ % MapCache::kEntries);
+  cache.keys[slot] = key;
+  cache.maps[slot] = *map;
+  return SP24_OK;
+}
+
+int sm_count() {
+  static std::atomic<int> known[64];
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+  const bool cacheable = dev >= 0 && dev < 64;
+  if (cacheable && (n = known[dev].load(std::memory_order_relaxed)) > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 1;
+  if (cacheable) known[dev].store(n, std::memory_order_relaxed);
   return n;
+}
+
+// Process-wide settings: the benchmarking overrides (environment, read once, or sp24_set_tile_override)
+// and the fault-path test hooks (sp24_test_set_fault_hooks only; never read from the environment).
+struct Settings {
+  std::atomic<int> ctas{0}, block_n{0}, mblk{0}, band{0}, log{0};
+  std::atomic<long long> test_wait_cycles{0};
+  std::atomic<int> test_skip_stage{0};
+};
+Settings& settings() {
+  static Settings st;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    if (const char* env = getenv("SP24_TILE")) {
+      int c = 0, n = 0, m = 1;
+      if (sscanf(env, "%dx%dx%d", &c, &n, &m) >= 2) { st.ctas = c; st.block_n = n; st.mblk = m; }
+    }
+    if (const char* env = getenv("SP24_BAND")) st.band = atoi(env) > 0 ? atoi(env) : 0;
+    if (const char* env = getenv("SP24_LOG")) st.log = atoi(env) != 0 || env[0] == '\0' ? 1 : 0;
+  });
+  return st;
 }
 
 template <int KIND, bool SPARSE, int BLOCK_N, int CTAS, int MBLK, bool B_MN>
@@ -988,13 +1050,15 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   p.cd_type = (int)d->cd_type;
   p.has_c = has_c ? 1 : 0;
   p.wait_limit = kWaitTimeoutCycles;
-  // Test hooks for the failure path (tests/test_gpu_timeout.py): a shorter limit, and a pipeline that
-  // stalls by leaving out one k-block.  Nothing faults or hangs: the waits expire and the kernel returns.
-  if (const char* env = getenv("SP24_TEST_WAIT_CYCLES")) {
-    const long long v = atoll(env);
+  // Test hooks for the failure path (set through sp24_test_set_fault_hooks only): a shorter limit, and a
+  // pipeline that stalls by leaving out one k-block.  Nothing faults or hangs: the waits expire and the
+  // kernel returns.
+  Settings& cfg = settings();
+  {
+    const long long v = cfg.test_wait_cycles.load(std::memory_order_relaxed);
     if (v >= 1000000) p.wait_limit = v;
+    p.test_skip_stage = cfg.test_skip_stage.load(std::memory_order_relaxed);
   }
-  if (const char* env = getenv("SP24_TEST_SKIP_STAGE")) p.test_skip_stage = atoi(env) != 0;
   p.cd_col_major = d->order_d == SP24_COL_MAJOR ? 1 : 0;
   const bool sparse = !d->a_is_dense;
   const bool i8 = d->ab_type == SP24_I8, tf32 = d->ab_type == SP24_F32, f8 = is_fp8(d->ab_type);
@@ -1015,16 +1079,14 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
     if (has_256 && d->N <= 2048 && (d->N + 255) / 256 < n_tiles) block_n = 256;
   }
   p.band = 16 / mblk;
-  if (const char* env = getenv("SP24_TILE")) {
-    int c = 0, n = 0, m = 1;
-    if (sscanf(env, "%dx%dx%d", &c, &n, &m) >= 2) { ctas = c; block_n = n; mblk = m; }
+  if (const int c = cfg.ctas.load(std::memory_order_relaxed)) {
+    ctas = c;
+    block_n = cfg.block_n.load(std::memory_order_relaxed);
+    mblk = cfg.mblk.load(std::memory_order_relaxed);
   }
-  if (const char* env = getenv("SP24_BAND")) {
-    int b = atoi(env);
-    if (b > 0) p.band = b;
-  }
+  if (const int b = cfg.band.load(std::memory_order_relaxed)) p.band = b;
   const bool b_mn = d->order_b == SP24_ROW_MAJOR;  // B stored N-contiguous
-  if (getenv("SP24_LOG"))
+  if (cfg.log.load(std::memory_order_relaxed))
     fprintf(stderr, "sp24_gemm: M=%lld N=%lld K=%lld ab=%d cd=%d %s%s tile=%dx%dx%d band=%d beta=%g%s%s\n", (long long)d->M,
             (long long)d->N, (long long)d->K, (int)d->ab_type, (int)d->cd_type, sparse ? "sparse" : "dense",
             b_mn ? " B:N-contiguous" : "", ctas, block_n, mblk, p.band, (double)fbeta, dq ? " dequant" : "",
@@ -1098,13 +1160,33 @@ extern "C" sp24_status sp24_conv3x3_nhwc(const sp24_gemm_desc* d, int64_t Nb, in
   return run_gemm(&dd, alpha, A, meta, x, beta, C, D, workspace, workspace_bytes, stream, nullptr, &cv);
 }
 
-extern "C" sp24_status sp24_gemm_status(const void* workspace, void* stream) {
+extern "C" sp24_status sp24_gemm_status(void* workspace, void* stream) {
   SP24_RETURN_IF(workspace == nullptr, SP24_ERR_NULL);
   uint32_t host[4] = {0, 0, 0, 0};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   SP24_CUDA_CHECK(cudaMemcpyAsync(host, workspace, sizeof(host), cudaMemcpyDeviceToHost, s));
   SP24_CUDA_CHECK(cudaStreamSynchronize(s));
-  return host[0] == 0 ? SP24_OK : SP24_ERR_TIMEOUT;
+  if (host[0] == 0) return SP24_OK;
+  // reported once: the record starts again from "ok" for the launches that follow
+  SP24_CUDA_CHECK(cudaMemsetAsync(workspace, 0, sizeof(host), s));
+  return SP24_ERR_TIMEOUT;
+}
+
+extern "C" sp24_status sp24_set_tile_override(int ctas, int block_n, int mblk, int band) {
+  SP24_RETURN_IF(ctas < 0 || block_n < 0 || mblk < 0 || band < 0, SP24_ERR_SHAPE);
+  Settings& cfg = settings();
+  cfg.block_n.store(ctas ? block_n : 0, std::memory_order_relaxed);
+  cfg.mblk.store(ctas ? (mblk ? mblk : 1) : 0, std::memory_order_relaxed);
+  cfg.ctas.store(ctas, std::memory_order_relaxed);
+  cfg.band.store(band, std::memory_order_relaxed);
+  return SP24_OK;
+}
+
+extern "C" sp24_status sp24_test_set_fault_hooks(long long wait_cycles, int skip_stage) {
+  Settings& cfg = settings();
+  cfg.test_wait_cycles.store(wait_cycles, std::memory_order_relaxed);
+  cfg.test_skip_stage.store(skip_stage ? 1 : 0, std::memory_order_relaxed);
+  return SP24_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1120,12 +1202,14 @@ extern "C" sp24_status sp24_gemm_status(const void* workspace, void* stream) {
 // The array's name is only a host-side stand-in in host code, not a device address, so the
 // address is resolved with cudaGetSymbolAddress once per device (with that device current) on
 // the first call made on that device; that first call should therefore come before any stream
-// capture.  The entry point calls no cudaMalloc, cudaFree or other allocating routine.
+// capture.  The entry points call no cudaMalloc, cudaFree or other allocating routine.
 //
-// All calls on a device share the one array, which keeps the previous call's contents; the
-// status word is cleared on the stream before each launch.  Calls that overlap on the GPU
-// (different streams) race on that word: serialise them, or use sp24_gemm with one workspace
-// per stream.
+// All calls on a device share the one array.  It starts out zero-filled (static storage) and the
+// kernels only ever write a non-zero code into it, so nothing has to be cleared between calls:
+// the record keeps the first expired wait of any call until sp24_gemm_static_ws_status reads and
+// clears it.  Calls that overlap on the GPU (different streams) share that one record, so a
+// reported timeout cannot be attributed to one of them: serialise them, or use sp24_gemm with
+// one workspace per stream.
 // ---------------------------------------------------------------------------------------------
 namespace {
 constexpr size_t kStaticWorkspaceBytes = 4096;  // stated maximum; sp24_gemm currently needs 256
@@ -1134,6 +1218,21 @@ static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspa
 constexpr int kMaxDevices = 64;
 std::mutex g_static_ws_mutex;
 void* g_static_ws_ptr[kMaxDevices] = {};
+
+// device address of the array on the current device (looked up once per device)
+sp24_status static_workspace(void** out) {
+  int dev = 0;
+  SP24_CUDA_CHECK(cudaGetDevice(&dev));
+  SP24_RETURN_IF(dev < 0 || dev >= kMaxDevices, SP24_ERR_UNSUPPORTED);
+  std::lock_guard<std::mutex> lock(g_static_ws_mutex);
+  if (g_static_ws_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || ptr == nullptr) return SP24_ERR_CUDA;
+    g_static_ws_ptr[dev] = ptr;
+  }
+  *out = g_static_ws_ptr[dev];
+  return SP24_OK;
+}
 }  // namespace
 
 extern "C" sp24_status sp24_gemm_static_ws(const sp24_gemm_desc* d, const void* alpha, const void* A,
@@ -1142,18 +1241,15 @@ extern "C" sp24_status sp24_gemm_static_ws(const sp24_gemm_desc* d, const void* 
   SP24_RETURN_IF(d == nullptr, SP24_ERR_NULL);
   // the problem's workspace need must fit the fixed array
   SP24_RETURN_IF(sp24_gemm_workspace_bytes(d) > kStaticWorkspaceBytes, SP24_ERR_WORKSPACE);
-  int dev = 0;
-  SP24_CUDA_CHECK(cudaGetDevice(&dev));
-  SP24_RETURN_IF(dev < 0 || dev >= kMaxDevices, SP24_ERR_UNSUPPORTED);
   void* ws = nullptr;
-  {
-    std::lock_guard<std::mutex> lock(g_static_ws_mutex);
-    if (g_static_ws_ptr[dev] == nullptr) {
-      void* ptr = nullptr;
-      if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || ptr == nullptr) return SP24_ERR_CUDA;
-      g_static_ws_ptr[dev] = ptr;
-    }
-    ws = g_static_ws_ptr[dev];
-  }
+  sp24_status st = static_workspace(&ws);
+  if (st != SP24_OK) return st;
   return sp24_gemm(d, alpha, A, meta, B, beta, C, D, ws, kStaticWorkspaceBytes, stream);
+}
+
+extern "C" sp24_status sp24_gemm_static_ws_status(void* stream) {
+  void* ws = nullptr;
+  sp24_status st = static_workspace(&ws);
+  if (st != SP24_OK) return st;
+  return sp24_gemm_status(ws, stream);
 }

@@ -644,9 +644,8 @@ static sp24_status validate_matrix_args(sp24_dtype t, int64_t M, int64_t K, int6
 using namespace sp24;
 
 // FP32 storage = the 1:2 pattern of the TF32 mode; vectorised paths only (16-byte aligned, K % 8 == 0).
-static sp24_status validate_f32(int64_t M, int64_t K, const void* a, int64_t lda, const void* b, int64_t ldb_bytes_ok) {
+static sp24_status validate_f32(int64_t M, int64_t K) {
   SP24_RETURN_IF(M < 0 || K < 0 || K % 8 != 0, SP24_ERR_SHAPE);
-  (void)a; (void)lda; (void)b; (void)ldb_bytes_ok;
   return SP24_OK;
 }
 
@@ -662,7 +661,7 @@ static dim3 f32_grid(int64_t units, int64_t rows, dim3& block) {
 extern "C" sp24_status sp24_prune(sp24_dtype t, int64_t M, int64_t K, const void* x, int64_t ldx, void* y,
                                   int64_t ldy, void* stream) {
   if (t == SP24_F32) {
-    sp24_status sf = validate_f32(M, K, x, ldx, y, ldy);
+    sp24_status sf = validate_f32(M, K);
     if (sf != SP24_OK) return sf;
     if (M == 0 || K == 0) return SP24_OK;
     SP24_RETURN_IF(x == nullptr || y == nullptr, SP24_ERR_NULL);
@@ -804,7 +803,7 @@ extern "C" sp24_status sp24_compress(sp24_dtype t, int64_t M, int64_t K, const v
                                      int64_t ldv, void* meta, sp24_meta_layout l, unsigned long long* dropped,
                                      void* stream) {
   if (t == SP24_F32) {
-    sp24_status sf = validate_f32(M, K, x, ldx, vals, ldv);
+    sp24_status sf = validate_f32(M, K);
     if (sf != SP24_OK) return sf;
     SP24_RETURN_IF(l != SP24_META_CANONICAL && l != SP24_META_TCGEN05, SP24_ERR_UNSUPPORTED);
     if (M == 0 || K == 0) return SP24_OK;
@@ -846,7 +845,7 @@ extern "C" sp24_status sp24_prune_compress(sp24_dtype t, int64_t M, int64_t K, c
 extern "C" sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals, int64_t ldv,
                                        const void* meta, sp24_meta_layout l, void* y, int64_t ldy, void* stream) {
   if (t == SP24_F32) {
-    sp24_status sf = validate_f32(M, K, vals, ldv, y, ldy);
+    sp24_status sf = validate_f32(M, K);
     if (sf != SP24_OK) return sf;
     SP24_RETURN_IF(l != SP24_META_CANONICAL && l != SP24_META_TCGEN05, SP24_ERR_UNSUPPORTED);
     if (M == 0 || K == 0) return SP24_OK;

@@ -37,3 +37,12 @@ def _built_library():
     except Exception as e:  # noqa: BLE001 - reported by the tests that need the library
         print(f"could not build libsp24.so: {e}", file=sys.stderr)
     yield
+
+
+@pytest.fixture
+def force_tile():
+    """force_tile("2x224x2") makes every GEMM call of the test use that tile shape; the automatic
+    choice is restored afterwards."""
+    from paper_2104_08378_b200 import binding
+    yield binding.set_tile_override
+    binding.set_tile_override(None)

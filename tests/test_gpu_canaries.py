@@ -70,7 +70,7 @@ def test_streaming_kernels_stay_inside_their_outputs(sp, dtype, shape):
 
 @pytest.mark.parametrize("kind", ["bf16", "i8", "e4m3", "tf32"])
 @pytest.mark.parametrize("tile", ["1x128x1", "2x224x1", "2x224x2"])
-def test_gemm_stays_inside_d(sp, monkeypatch, kind, tile):
+def test_gemm_stays_inside_d(sp, force_tile, kind, tile):
     M, N, K = 1184, 736, 640
     if kind == "i8":
         A = torch.randint(-127, 128, (M, K), dtype=torch.int8, device="cuda")
@@ -85,7 +85,7 @@ def test_gemm_stays_inside_d(sp, monkeypatch, kind, tile):
         A, Bt, cd, cdt = torch.randn(M, K, device="cuda").bfloat16(), torch.randn(N, K, device="cuda").bfloat16(), "bf16", torch.bfloat16
     vals, meta, _ = sp.compress(A)
     ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
-    monkeypatch.setenv("SP24_TILE", tile)
+    force_tile(tile)
     for ld_extra in (0, 32):
         D = Guarded(M, N, cdt, N + ld_extra)
         sp.gemm(vals, meta, Bt, out=D.t, cd=cd, ws=ws)

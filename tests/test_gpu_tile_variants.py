@@ -1,7 +1,7 @@
 """Every tile shape the GEMM is built in, for every operand kind, against the oracle.
 
 The library picks the tile shape from the problem size, so at sizes the oracle finishes in seconds
-only the small shapes would run; SP24_TILE=<CTAs>x<BLOCK_N>x<m-blocks> (read on every call)
+only the small shapes would run; sp24_set_tile_override(<CTAs>, <BLOCK_N>, <m-blocks>)
 forces each one.  Sizes span several tiles with ragged tails in M and N."""
 import numpy as np
 import pytest
@@ -36,14 +36,14 @@ def _dev(a, kind):
 @pytest.mark.parametrize("dense", [False, True])
 @pytest.mark.parametrize("tile", TILES)
 @pytest.mark.parametrize("kind", ["bf16", "f16", "i8", "tf32", "e4m3", "e5m2"])
-def test_forced_tile_shape(sp, monkeypatch, kind, tile, dense):
+def test_forced_tile_shape(sp, force_tile, kind, tile, dense):
     if tile not in BUILT[kind]:
         pytest.skip("shape not built for this kind")
     M, N, K = 1184, 736, 640          # 2.3 tiles of 512 rows, 3.3 of 224 columns, 5 k-blocks of 128
     A = inputs._matrix(("int8",) if kind == "i8" else ("normal", 1.0), kind, 21, 5, K, 0, M)
     Bt = inputs._matrix(("int8",) if kind == "i8" else ("uniform", -1.0, 1.0), kind, 22, 6, K, 0, N)
     Ad, Btd = _dev(A, kind), _dev(Bt, kind)
-    monkeypatch.setenv("SP24_TILE", tile)
+    force_tile(tile)
     if kind == "i8":
         Cm = inputs._matrix(("int8",), "i8", 23, 7, N, 0, M).astype(np.int32)
         Cd, alpha, beta, cd = torch.from_numpy(Cm).cuda(), 1, 1, "i32"

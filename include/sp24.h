@@ -144,10 +144,10 @@ sp24_status sp24_decompress(sp24_dtype t, int64_t M, int64_t K, const void* vals
 
 /* Problem description of D = alpha * op(A) * B + beta * C  (Section 3.2, Figure 2).
  *   ab_type: SP24_F16 or SP24_BF16 (FP32 accumulate), SP24_I8 (INT32 accumulate) or SP24_F32
- *            (TF32 mode, 1:2 pattern, FP32 accumulate; cd_type SP24_F32 and K-contiguous B
- *            only; inputs are used with their low 13 mantissa bits ignored) -- the
- *            operand/accumulator pairs of Table 1.  SP24_E4M3 or SP24_E5M2 (both operands the
- *            same type, FP32 accumulate, K-contiguous B only) go beyond that table.
+ *            (TF32 mode, 1:2 pattern, FP32 accumulate; cd_type SP24_F32 only; inputs are used
+ *            with their low 13 mantissa bits ignored) -- the operand/accumulator pairs of
+ *            Table 1 (its FP16-accumulate row is sp24_gemm_f16acc).  SP24_E4M3 or SP24_E5M2
+ *            (both operands the same type, FP32 accumulate) go beyond that table.
  *   cd_type: type of C and D.  F16/BF16 operands: SP24_F16, SP24_BF16 (ab_type's own) or
  *            SP24_F32.  I8 operands: SP24_I32.  E4M3/E5M2 operands: SP24_F16, SP24_BF16 or
  *            SP24_F32.
@@ -194,6 +194,22 @@ size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d);
 sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A,
                       const void* meta, const void* B, const void* beta, const void* C,
                       void* D, void* workspace, size_t workspace_bytes, void* stream);
+
+/* The FP16-accumulation mode of Table 1 (FP16 operands, FP16 accumulator; Section 3.2): sp24_gemm
+ * with the tensor cores adding the products into a binary16 accumulator instead of an FP32 one.
+ *   d->ab_type must be SP24_F16; d->cd_type SP24_F16 or SP24_F32; everything else as for sp24_gemm
+ *   (sparse or dense variant, both orders of B, C and D; alpha, beta and C are applied in FP32 to
+ *   the widened accumulator).
+ * Accuracy: the running sum is rounded to binary16 after every tensor-core instruction (32 values of
+ * K for the sparse form, 16 for the dense one), so the error grows with K:
+ * |err| <= (K/32 + 2) * 2^-10 * (|A|.|B|)_ij is the bound the tests use, against 2^-11 relative for
+ * one final rounding with sp24_gemm.  On these tensor cores a binary16 accumulator occupies a full
+ * 32-bit cell of tensor memory and the instruction rate is that of FP32 accumulation, so the mode
+ * buys no speed here (measured; see the benchmark's other_configs): it exists for bit-compatibility
+ * with deployments that used it. */
+sp24_status sp24_gemm_f16acc(const sp24_gemm_desc* d, const void* alpha, const void* A,
+                             const void* meta, const void* B, const void* beta, const void* C,
+                             void* D, void* workspace, size_t workspace_bytes, void* stream);
 
 /* INT8 sparse GEMM with a dequantising epilogue, for the deployment the paper describes in
  * Section 4.4 and Section 5.1: INT8 weights and activations, per-row scaling factors for the

@@ -32,7 +32,7 @@ EXPORTS = [
     "sp24_decompress", "sp24_prune_compress", "sp24_gemm_workspace_bytes", "sp24_gemm", "sp24_gemm_status",
     "sp24_im2col_nhwc_3x3", "sp24_pipeline_host", "sp24_gemm_static_ws", "sp24_gemm_i8_dequant",
     "sp24_conv3x3_nhwc", "sp24_kept_magnitude", "sp24_apply_mask", "sp24_prune_2d",
-    "sp24_gemm_static_ws_status", "sp24_set_tile_override", "sp24_test_set_fault_hooks",
+    "sp24_gemm_static_ws_status", "sp24_set_tile_override", "sp24_test_set_fault_hooks", "sp24_gemm_f16acc",
 ]
 
 
@@ -70,6 +70,8 @@ def _load() -> ctypes.CDLL:
     lib.sp24_gemm_workspace_bytes.argtypes = [ctypes.POINTER(GemmDesc)]
     lib.sp24_gemm_workspace_bytes.restype = sz
     lib.sp24_gemm.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sp24_gemm_f16acc.argtypes = lib.sp24_gemm.argtypes
+    lib.sp24_gemm_f16acc.restype = ci
     lib.sp24_gemm_static_ws.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sp24_gemm_static_ws.restype = ci
     lib.sp24_gemm_i8_dequant.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, ci, ctypes.c_float, vp, vp,
@@ -215,10 +217,10 @@ def workspace(device) -> torch.Tensor:
 def gemm(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor, *, alpha=1.0, beta=0.0,
          C: torch.Tensor | None = None, out: torch.Tensor | None = None, cd: str | None = None,
          ab: str | None = None, a_is_dense: bool = False, ws: torch.Tensor | None = None,
-         b_row_major: bool = False, cd_col_major: bool = False) -> torch.Tensor:
-    """sp24_gemm.  A: vals [M, K/2] (or dense [M, K]); Bt: [N, K] (K contiguous), or with
-    b_row_major=True the K x N matrix itself, [K, N] (N contiguous); C/D: [M, N], or with
-    cd_col_major=True their transposes [N, M] (M contiguous)."""
+         b_row_major: bool = False, cd_col_major: bool = False, acc_f16: bool = False) -> torch.Tensor:
+    """sp24_gemm (sp24_gemm_f16acc with acc_f16=True).  A: vals [M, K/2] (or dense [M, K]); Bt: [N, K]
+    (K contiguous), or with b_row_major=True the K x N matrix itself, [K, N] (N contiguous); C/D: [M, N],
+    or with cd_col_major=True their transposes [N, M] (M contiguous)."""
     ab = _dtype_of(A, ab)
     M = A.shape[0]
     K = A.shape[1] if a_is_dense else 2 * A.shape[1]
@@ -232,8 +234,10 @@ def gemm(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor, *, alpha=
                      C.stride(0) if C is not None else (M if cd_col_major else N), out.stride(0), a_is_dense,
                      b_row_major, cd_col_major)
     a, b = _scalar(ab, alpha), _scalar(ab, beta)
-    _check(lib.sp24_gemm(ctypes.byref(desc), ctypes.byref(a), _ptr(A), _ptr(meta), _ptr(Bt),
-                         ctypes.byref(b), _ptr(C), _ptr(out), _ptr(ws), ws.numel(), _stream()), "sp24_gemm")
+    fn = lib.sp24_gemm_f16acc if acc_f16 else lib.sp24_gemm
+    _check(fn(ctypes.byref(desc), ctypes.byref(a), _ptr(A), _ptr(meta), _ptr(Bt),
+              ctypes.byref(b), _ptr(C), _ptr(out), _ptr(ws), ws.numel(), _stream()),
+           "sp24_gemm_f16acc" if acc_f16 else "sp24_gemm")
     return out
 
 

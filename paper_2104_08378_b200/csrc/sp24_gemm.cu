@@ -66,6 +66,7 @@ struct GemmParams {
   // int8 dequantising epilogue (sp24_gemm_i8_dequant): out = act(row_scale[i] * acc + bias[i]),
   // requantised with out_inv_scale when the output type is int8
   int32_t dequant, relu;
+  int32_t acc_f16;    // FP16 accumulation (kind::f16 with a binary16 accumulator; FP16 operands only)
   const float* row_scale;
   const float* bias;
   float out_inv_scale;
@@ -90,6 +91,9 @@ struct Cfg {
   static constexpr int kBChunks = (kBRows + kBChunkElems - 1) / kBChunkElems;
   static constexpr int kBChunkBytes = kKPerStage * kAtomBytes;
   static constexpr int kBKStepBytes = (SPARSE ? 2 : 1) * (kAtomElems / 4) * kAtomBytes;  // k-rows of one MMA
+  // an MN-major tf32 operand exists only in the 128-byte swizzle with 32-byte units (groups of 4 k-rows)
+  static constexpr uint32_t kBMnLayout = KIND == 2 ? ptx::kLayoutSw128Base32 : ptx::kLayoutSw128;
+  static constexpr uint32_t kBMnSbo = KIND == 2 ? 512 : 1024;
   static constexpr int kBBytes = B_MN ? kBChunks * kBChunkBytes : kBBoxes * kBRows * kAtomBytes;
   static constexpr int kEBlocks = SPARSE ? (one_byte_operands(KIND) ? 2 : 1) : 0;  // 2048-byte metadata blocks per m-block and stage
   static constexpr int kEBlockBytes = kEBlocks * 2048;
@@ -153,10 +157,10 @@ __device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int
 }
 
 template <int KIND>
-__device__ __forceinline__ uint32_t make_idesc(bool sparse, bool b_mn_major, int a_fmt, int m, int n) {
+__device__ __forceinline__ uint32_t make_idesc(bool sparse, bool b_mn_major, int a_fmt, int m, int n, bool acc_f16) {
   uint32_t d = 0;
   d |= (sparse ? 1u : 0u) << 2;
-  d |= (KIND == 1 ? 2u : 1u) << 4;                 // accumulator: int32 / fp32
+  d |= (KIND == 1 ? 2u : (acc_f16 ? 0u : 1u)) << 4;  // accumulator: int32 / fp32 / fp16
   // kind f16: f16 = 0, bf16 = 1; tf32: 2; int8: 1 = signed; 8-bit floats: e4m3 = 0, e5m2 = 1
   uint32_t fmt = (KIND == 0 || KIND == 3) ? (uint32_t)a_fmt : (KIND == 1 ? 1u : 2u);
   d |= fmt << 7;
@@ -168,15 +172,6 @@ __device__ __forceinline__ uint32_t make_idesc(bool sparse, bool b_mn_major, int
 }
 
 // ---- epilogue helpers ----------------------------------------------------------------------------
-// A staging buffer holds one 32-row x 32-column box of C / D in the layout the TMA uses: rows of 64
-// bytes with the 64-byte swizzle (2-byte types) or rows of 128 bytes with the 128-byte swizzle
-// (4-byte types).  16-byte unit v of row r sits at unit v ^ ((r >> 1) & 3), resp. v ^ (r & 7), which
-// also keeps the row-per-thread accesses below free of bank conflicts.
-__device__ __forceinline__ uint4* staged_unit(uint8_t* buf, int cs, int row, int v) {
-  return cs == 2 ? reinterpret_cast<uint4*>(buf + row * 64 + ((v ^ ((row >> 1) & 3)) << 4))
-                 : reinterpret_cast<uint4*>(buf + row * 128 + ((v ^ (row & 7)) << 4));
-}
-
 // Dequantising epilogue of the int8 path, all in fp32 and in exactly this order (the int8 output
 // is compared bit for bit): t = float(acc) (round to nearest), y = fma(scale, t, bias), optional
 // max(y, 0); int8 output: round-to-nearest-even of y * out_inv_scale, clamped to [-127, 127].
@@ -189,51 +184,85 @@ __device__ __forceinline__ int requant_i8(float y, float inv) {
   return max(-127, min(127, q));
 }
 
-__device__ __forceinline__ void convert_row_dequant(const uint32_t (&r)[32], uint8_t* buf, int lane, const GemmParams& p,
-                                                    float scale, float bias) {
-  if (p.cd_type == SP24_F32) {
+__device__ __forceinline__ uint32_t pack_16bit(float lo, float hi, bool bf) {
+  if (bf) {
+    __nv_bfloat162 o = __float22bfloat162_rn(make_float2(lo, hi));
+    return *reinterpret_cast<uint32_t*>(&o);
+  }
+  __half2 o = __float22half2_rn(make_float2(lo, hi));
+  return *reinterpret_cast<uint32_t*>(&o);
+}
+__device__ __forceinline__ float2 unpack_16bit(uint32_t w, bool bf) {
+  return bf ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w))
+            : __half22float2(*reinterpret_cast<const __half2*>(&w));
+}
+
+// One thread's row of a 32-column box: out = alpha * acc + beta * c (or the dequantising form) as
+// the packed words of the output row: 16 words for 2-byte outputs (CS = 2), 32 for 4-byte ones.
+// `c` holds the row's C values in the same packing and is read only if has_c.  One multiply and
+// one fused multiply-add per element, whichever path stores the row.
+template <int KIND, int CS>
+__device__ __forceinline__ void compute_row(const uint32_t (&r)[32], const uint32_t (&c)[8 * CS], bool has_c,
+                                            const GemmParams& p, float scale, float bias, uint32_t (&o)[8 * CS]) {
+  const bool bf = p.cd_type == SP24_BF16;
+  if constexpr (CS == 4) {
+    if (KIND == 1 && p.dequant) {
 #pragma unroll
-    for (int v = 0; v < 8; ++v) {
-      float4 o = make_float4(dequant_value(r[4 * v], scale, bias, p.relu), dequant_value(r[4 * v + 1], scale, bias, p.relu),
-                             dequant_value(r[4 * v + 2], scale, bias, p.relu), dequant_value(r[4 * v + 3], scale, bias, p.relu));
-      *reinterpret_cast<float4*>(staged_unit(buf, 4, lane, v)) = o;
-    }
-  } else if (p.cd_type == SP24_I8) {
-    // rows of 32 bytes, no swizzle
+      for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(dequant_value(r[e], scale, bias, p.relu));
+    } else if (KIND == 1) {
 #pragma unroll
-    for (int v = 0; v < 2; ++v) {
-      uint32_t w[4];
+      for (int e = 0; e < 32; ++e) o[e] = r[e] + (has_c ? c[e] : 0u);
+    } else {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        uint32_t word = 0;
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          int q = requant_i8(dequant_value(r[16 * v + 4 * e + b], scale, bias, p.relu), p.out_inv_scale);
-          word |= ((uint32_t)q & 0xFFu) << (8 * b);
-        }
-        w[e] = word;
+      for (int e = 0; e < 32; ++e) {
+        float f = __fmul_rn(p.alpha, __uint_as_float(r[e]));
+        if (has_c) f = __fmaf_rn(p.beta, __uint_as_float(c[e]), f);
+        o[e] = __float_as_uint(f);
       }
-      *reinterpret_cast<uint4*>(buf + lane * 32 + v * 16) = make_uint4(w[0], w[1], w[2], w[3]);
     }
   } else {
-    const bool bf = p.cd_type == SP24_BF16;
+    if (KIND == 1) {  // dequantised to a 16-bit type (the plain int8 GEMM writes 4-byte results)
 #pragma unroll
-    for (int v = 0; v < 4; ++v) {
-      uint32_t ow[4];
+      for (int e = 0; e < 16; ++e)
+        o[e] = pack_16bit(dequant_value(r[2 * e], scale, bias, p.relu), dequant_value(r[2 * e + 1], scale, bias, p.relu), bf);
+    } else {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        float2 f = make_float2(dequant_value(r[8 * v + 2 * e], scale, bias, p.relu),
-                               dequant_value(r[8 * v + 2 * e + 1], scale, bias, p.relu));
-        if (bf) {
-          __nv_bfloat162 o = __float22bfloat162_rn(f);
-          ow[e] = *reinterpret_cast<uint32_t*>(&o);
-        } else {
-          __half2 o = __float22half2_rn(f);
-          ow[e] = *reinterpret_cast<uint32_t*>(&o);
+      for (int e = 0; e < 16; ++e) {
+        float f0 = __fmul_rn(p.alpha, __uint_as_float(r[2 * e])), f1 = __fmul_rn(p.alpha, __uint_as_float(r[2 * e + 1]));
+        if (has_c) {
+          const float2 g = unpack_16bit(c[e], bf);
+          f0 = __fmaf_rn(p.beta, g.x, f0);
+          f1 = __fmaf_rn(p.beta, g.y, f1);
         }
+        o[e] = pack_16bit(f0, f1, bf);
       }
-      *staged_unit(buf, 2, lane, v) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
     }
+  }
+}
+
+// FP16 accumulation: every accumulator cell of tensor memory holds a binary16 value in its low half
+__device__ __forceinline__ void widen_f16_accumulators(uint32_t (&r)[32]) {
+#pragma unroll
+  for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__half2float(__ushort_as_half((unsigned short)(r[e] & 0xFFFFu))));
+}
+
+// int8 output of the dequantising epilogue: rows of 32 bytes, no swizzle
+__device__ __forceinline__ void convert_row_dequant_i8(const uint32_t (&r)[32], uint8_t* buf, int lane, const GemmParams& p,
+                                                       float scale, float bias) {
+#pragma unroll
+  for (int v = 0; v < 2; ++v) {
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      uint32_t word = 0;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        int q = requant_i8(dequant_value(r[16 * v + 4 * e + b], scale, bias, p.relu), p.out_inv_scale);
+        word |= ((uint32_t)q & 0xFFu) << (8 * b);
+      }
+      w[e] = word;
+    }
+    *reinterpret_cast<uint4*>(buf + lane * 32 + v * 16) = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
 
@@ -256,64 +285,6 @@ __device__ __forceinline__ void convert_row_dequant_transposed(const uint32_t (&
         __half o = __float2half_rn(y);
         *u = *reinterpret_cast<uint16_t*>(&o);
       }
-    }
-  }
-}
-
-// This thread's row of the box: out = alpha * acc + beta * c, written over c in the staging buffer.
-template <int KIND>
-__device__ __forceinline__ void convert_row(const uint32_t (&r)[32], uint8_t* buf, int lane, const GemmParams& p) {
-  if (KIND == 1) {
-#pragma unroll
-    for (int v = 0; v < 8; ++v) {
-      uint4* u = staged_unit(buf, 4, lane, v);
-      uint4 o = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
-      if (p.has_c) { uint4 c = *u; o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w; }
-      *u = o;
-    }
-  } else if (p.cd_type == SP24_F32) {
-#pragma unroll
-    for (int v = 0; v < 8; ++v) {
-      uint4* u = staged_unit(buf, 4, lane, v);
-      float4 o = make_float4(p.alpha * __uint_as_float(r[4 * v]), p.alpha * __uint_as_float(r[4 * v + 1]),
-                             p.alpha * __uint_as_float(r[4 * v + 2]), p.alpha * __uint_as_float(r[4 * v + 3]));
-      if (p.has_c) {
-        float4 c = *reinterpret_cast<float4*>(u);
-        o.x += p.beta * c.x; o.y += p.beta * c.y; o.z += p.beta * c.z; o.w += p.beta * c.w;
-      }
-      *reinterpret_cast<float4*>(u) = o;
-    }
-  } else {
-    const bool bf = p.cd_type == SP24_BF16;
-#pragma unroll
-    for (int v = 0; v < 4; ++v) {
-      uint4* u = staged_unit(buf, 2, lane, v);
-      float f[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) f[e] = p.alpha * __uint_as_float(r[8 * v + e]);
-      if (p.has_c) {
-        uint4 c = *u;
-        const uint32_t cw[4] = {c.x, c.y, c.z, c.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float2 g = bf ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&cw[e]))
-                        : __half22float2(*reinterpret_cast<const __half2*>(&cw[e]));
-          f[2 * e] += p.beta * g.x;
-          f[2 * e + 1] += p.beta * g.y;
-        }
-      }
-      uint32_t ow[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (bf) {
-          __nv_bfloat162 o = __float22bfloat162_rn(make_float2(f[2 * e], f[2 * e + 1]));
-          ow[e] = *reinterpret_cast<uint32_t*>(&o);
-        } else {
-          __half2 o = __float22half2_rn(make_float2(f[2 * e], f[2 * e + 1]));
-          ow[e] = *reinterpret_cast<uint32_t*>(&o);
-        }
-      }
-      *u = make_uint4(ow[0], ow[1], ow[2], ow[3]);
     }
   }
 }
@@ -348,6 +319,134 @@ __device__ __forceinline__ void convert_row_transposed(const uint32_t (&r)[32], 
         *u = *reinterpret_cast<uint16_t*>(&o);
       }
     }
+  }
+}
+
+// ---- epilogue for row-major C / D of 2- or 4-byte elements ------------------------------------
+// The epilogue warps move C and D themselves.  C: every thread loads the 32 values of ITS
+// accumulator row straight from global memory into registers, the first boxes of a tile before
+// the tile's accumulators are even complete, the later ones a few boxes ahead, so that no load
+// latency is left on the path that holds the accumulators (tensor memory cannot be handed back to
+// the MMA issuer before it is drained).  D: the row is converted in registers, written to a small
+// per-warp buffer in shared memory and read back transposed, so that the global stores of a warp
+// cover whole 64-byte row segments.  A "pass" is 32 rows x 64 bytes (2 KB): a whole box of a 2-byte
+// type, half a box of a 4-byte type.
+template <int KIND, int CS, int BLOCK_N, int CTAS, int MBLK, int ACC_STAGES>
+__device__ __forceinline__ void epilogue_rows(const GemmParams& p, Shared* sh, uint8_t* epi, uint32_t tmem_base,
+                                              int cta_rank, int cluster_id, int num_clusters, int num_tiles, int warp,
+                                              int lane) {
+  constexpr int kSub = BLOCK_N / 32, kIters = MBLK * kSub;
+  constexpr int kBoxes = (kIters + 1) / 2;  // boxes per warp and tile (the two warps of a lane quarter alternate)
+  constexpr int W = 8 * CS;                 // 32-bit words of one box row
+  constexpr int P = CS == 2 ? 4 : 1;        // boxes whose C values are held in registers
+  constexpr int kPasses = CS / 2;
+  constexpr int kUnitElems = 16 / CS;       // elements per 16-byte unit
+  const int q = warp & 3, ew = warp - 2, half = ew >> 2;
+  const int nbuf = p.epi_bytes >= kEpiWarps * 4096 ? 2 : 1;
+  uint8_t* stage = epi + ew * (nbuf * 2048);
+  const uint8_t* Cb = static_cast<const uint8_t*>(p.C);
+  uint8_t* Db = static_cast<uint8_t*>(p.D);
+  const size_t ldc_b = (size_t)p.ldc * CS, ldd_b = (size_t)p.ldd * CS;
+  const int M = (int)p.M, N = (int)p.N;
+  const bool has_c = p.has_c != 0;
+  uint32_t creg[P][W];
+  int acc = 0;
+  uint32_t acc_phase = 0, pass_no = 0;
+  for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
+    int mt, nt;
+    tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
+    // box n of this warp in this tile: first row / column, accumulator column, inside the matrix?
+    auto geom = [&](int n, int& row0, int& col0, int& tcol) -> bool {
+      const int it = half + 2 * n;
+      const int j = it / kSub, sc = it - j * kSub;
+      row0 = ((mt * MBLK + j) * CTAS + cta_rank) * kBlockM + q * 32;
+      col0 = nt * BLOCK_N + sc * 32;
+      tcol = j * BLOCK_N + sc * 32;
+      return it < kIters && row0 < M && col0 < N;
+    };
+    auto load_c = [&](int n, uint32_t (&c)[W]) {
+      int row0, col0, tcol;
+      if (!geom(n, row0, col0, tcol)) return;
+      const int row = row0 + lane;
+      if (row >= M) return;
+      const uint4* src = reinterpret_cast<const uint4*>(Cb + (size_t)row * ldc_b + (size_t)col0 * CS);
+#pragma unroll
+      for (int v = 0; v < W / 4; ++v) {
+        if (col0 + v * kUnitElems < N) {
+          const uint4 x = src[v];
+          c[4 * v] = x.x; c[4 * v + 1] = x.y; c[4 * v + 2] = x.z; c[4 * v + 3] = x.w;
+        }
+      }
+    };
+    if (has_c) {
+#pragma unroll
+      for (int n = 0; n < P; ++n)
+        if (n < kBoxes) load_c(n, creg[n]);
+    }
+    if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u, p.wait_limit)) break;
+    ptx::tc_fence_after();
+    const uint32_t t_acc = tmem_base + (acc * MBLK) * BLOCK_N + ((uint32_t)(q * 32) << 16);
+    uint32_t racc[2][32];
+    {
+      int row0, col0, tcol;
+      geom(0, row0, col0, tcol);
+      ptx::tmem_ld_32x32b_x32(t_acc + tcol, racc[0]);
+    }
+#pragma unroll
+    for (int n = 0; n < kBoxes; ++n) {
+      if (half + 2 * n >= kIters) break;  // same answer for the whole warp
+      ptx::tmem_ld_wait();
+      if (half + 2 * (n + 1) < kIters) {
+        int row1, col1, tcol1;
+        geom(n + 1, row1, col1, tcol1);
+        ptx::tmem_ld_32x32b_x32(t_acc + tcol1, racc[(n + 1) & 1]);
+      } else {
+        // this warp's part of the accumulators is in registers: hand it back to the MMA issuer (CTA 0 of the pair)
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if (CTAS == 1) ptx::mbar_arrive(&sh->tmem_empty[acc]);
+          else ptx::mbar_arrive_cluster(&sh->tmem_empty[acc], 0);
+        }
+      }
+      int row0, col0, tcol;
+      const bool live = geom(n, row0, col0, tcol);  // same answer for the whole warp
+      uint32_t o[W];
+      if (live) {
+        uint32_t (&r)[32] = racc[n & 1];
+        if (KIND == 0 && p.acc_f16) widen_f16_accumulators(r);
+        float scale = 1.f, bias = 0.f;
+        if (KIND == 1 && p.dequant) {
+          const int row = min(row0 + lane, M - 1);
+          scale = __ldg(p.row_scale + row);
+          bias = p.bias ? __ldg(p.bias + row) : 0.f;
+        }
+        compute_row<KIND, CS>(r, creg[n % P], has_c, p, scale, bias, o);
+      }
+      // the C registers of box n are free: fetch box n + P into them (also when box n lies outside the matrix)
+      if (has_c && n + P < kBoxes) load_c(n + P, creg[n % P]);
+      if (live) {
+#pragma unroll
+        for (int ps = 0; ps < kPasses; ++ps) {
+          uint8_t* buf = stage + (nbuf == 2 ? (pass_no & 1u) * 2048 : 0);
+          if (nbuf == 1) __syncwarp();  // the reads of the previous pass are done
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            *reinterpret_cast<uint4*>(buf + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4)) =
+                make_uint4(o[16 * ps + 4 * u], o[16 * ps + 4 * u + 1], o[16 * ps + 4 * u + 2], o[16 * ps + 4 * u + 3]);
+          __syncwarp();
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int i = lane + 32 * k, rr = i >> 2, u = i & 3;
+            const uint4 x = *reinterpret_cast<const uint4*>(buf + rr * 64 + ((u ^ ((rr >> 1) & 3)) << 4));
+            const int grow = row0 + rr, gcol = col0 + ps * (64 / CS) + u * kUnitElems;
+            if (grow < M && gcol < N) *reinterpret_cast<uint4*>(Db + (size_t)grow * ldd_b + (size_t)gcol * CS) = x;
+          }
+          ++pass_no;
+        }
+      }
+    }
+    if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
   }
 }
 
@@ -499,7 +598,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int n_eff = min(BLOCK_N, (int)(p.N - (int64_t)nt * BLOCK_N));
         const int live = min(MBLK, (int)((p.M - (int64_t)mt * MBLK * CTAS * kBlockM + CTAS * kBlockM - 1) /
                                          (CTAS * kBlockM)));
-        const uint32_t idesc = make_idesc<KIND>(SPARSE, B_MN, p.a_fmt, kBlockM * CTAS, n_eff);
+        const uint32_t idesc = make_idesc<KIND>(SPARSE, B_MN, p.a_fmt, kBlockM * CTAS, n_eff, KIND == 0 && p.acc_f16);
         if (!bounded_wait(&sh->tmem_empty[acc], acc_phase ^ 1u, sh, p.status, 2u, p.wait_limit)) break;
         ptx::tc_fence_after();
         bool ok = true;
@@ -519,7 +618,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
               for (int i = 0; i < C::kEBlocks; ++i)
                 ptx::tmem_cp_128x128b<CTAS>(e_base + j * 8 + 4 * i,
-                                            ptx::smem_desc(se + j * C::kEBlockBytes + i * 2048, false, 128));
+                                            ptx::smem_desc(se + j * C::kEBlockBytes + i * 2048, ptx::kLayoutNone, 128));
             }
           }
 #pragma unroll
@@ -533,9 +632,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               const uint32_t accumulate = (kb > 0 || k > 0) ? 1u : 0u;
               if (SPARSE) {
                 // 32 bytes of compressed A and 64 bytes of B per instruction
-                uint64_t da = ptx::smem_desc(saj + k * 32, true, 1024);
-                uint64_t db = B_MN ? ptx::smem_desc(sb + k * C::kBKStepBytes, true, 1024, C::kBChunkBytes)
-                                   : ptx::smem_desc(sb + (k >> 1) * C::kBRows * kAtomBytes + (k & 1) * 64, true, 1024);
+                uint64_t da = ptx::smem_desc(saj + k * 32, ptx::kLayoutSw128, 1024);
+                uint64_t db = B_MN ? ptx::smem_desc(sb + k * C::kBKStepBytes, C::kBMnLayout, C::kBMnSbo, C::kBChunkBytes)
+                                   : ptx::smem_desc(sb + (k >> 1) * C::kBRows * kAtomBytes + (k & 1) * 64, ptx::kLayoutSw128, 1024);
                 if (!one_byte_operands(KIND)) {
                   // one 32-bit metadata column per instruction: even-aligned address + selector
                   ptx::mma_sparse<KIND, CTAS>(d_tmem, da, db, e_tmem + (k & ~1), idesc | (uint32_t)(k & 1), accumulate);
@@ -543,9 +642,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                   ptx::mma_sparse<KIND, CTAS>(d_tmem, da, db, e_tmem + 2 * k, idesc, accumulate);
                 }
               } else {
-                uint64_t da = ptx::smem_desc(saj + (k >> 2) * kBlockM * kAtomBytes + (k & 3) * 32, true, 1024);
-                uint64_t db = B_MN ? ptx::smem_desc(sb + k * C::kBKStepBytes, true, 1024, C::kBChunkBytes)
-                                   : ptx::smem_desc(sb + (k >> 2) * C::kBRows * kAtomBytes + (k & 3) * 32, true, 1024);
+                uint64_t da = ptx::smem_desc(saj + (k >> 2) * kBlockM * kAtomBytes + (k & 3) * 32, ptx::kLayoutSw128, 1024);
+                uint64_t db = B_MN ? ptx::smem_desc(sb + k * C::kBKStepBytes, C::kBMnLayout, C::kBMnSbo, C::kBChunkBytes)
+                                   : ptx::smem_desc(sb + (k >> 2) * C::kBRows * kAtomBytes + (k & 3) * 32, ptx::kLayoutSw128, 1024);
                 ptx::mma_dense<KIND, CTAS>(d_tmem, da, db, idesc, accumulate);
               }
             }
@@ -563,12 +662,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     }
   } else {
     // ------------------------------ epilogue ------------------------------
-    // Each warp owns 32 accumulator rows and walks its tiles in 32 x 32 boxes: TMA load of the C box
-    // (if beta != 0) into a staging buffer a few boxes ahead, tcgen05.ld of the accumulator columns,
-    // convert in place, TMA store of the D box.  Boxes outside the matrix are clipped by the TMA.
+    const int cs = elem_bytes((sp24_dtype)p.cd_type);
+    if (!p.cd_col_major && cs != 1) {
+      // row-major C / D: loads and stores by the epilogue warps themselves
+      if (KIND != 2 && cs == 2)
+        epilogue_rows<KIND, 2, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id,
+                                                                   num_clusters, num_tiles, warp, lane);
+      else
+        epilogue_rows<KIND, 4, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id,
+                                                                   num_clusters, num_tiles, warp, lane);
+    } else {
+    // Column-major C / D and 1-byte outputs.  Each warp owns 32 accumulator rows and walks its tiles in
+    // 32 x 32 boxes: TMA load of the C box (if beta != 0) into a staging buffer a few boxes ahead,
+    // tcgen05.ld of the accumulator columns, convert in place, TMA store of the D box.  Boxes outside
+    // the matrix are clipped by the TMA.
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
     const int ew = warp - 2;  // epilogue warp 0..7: warps ew and ew + 4 share a lane quarter
-    const int cs = elem_bytes((sp24_dtype)p.cd_type);
     const int buf_bytes = 1024 * cs;
     // Both warps of a quarter work (alternate boxes) when each can have a staging buffer of its own;
     // otherwise the second one only takes part in handing the accumulators back.
@@ -649,16 +758,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int b = seq % nbuf;
         uint8_t* buf = my_bufs + b * buf_bytes;
         if (p.has_c && !bounded_wait(&sh->c_full[ew][b], (seq / nbuf) & 1u, sh, p.status, 5u, p.wait_limit)) { ok = false; break; }
+        if (KIND == 0 && p.acc_f16) widen_f16_accumulators(r);
         if (KIND == 1 && p.dequant) {
           // this thread's output row: its scale and bias
           const int row = min(row0 + lane, (int)p.M - 1);
           const float scale = __ldg(p.row_scale + row), bias = p.bias ? __ldg(p.bias + row) : 0.f;
           if (p.cd_col_major) convert_row_dequant_transposed(r, buf, lane, p, scale, bias);
-          else convert_row_dequant(r, buf, lane, p, scale, bias);
-        } else if (p.cd_col_major) {
-          convert_row_transposed<KIND>(r, buf, lane, p);
+          else convert_row_dequant_i8(r, buf, lane, p, scale, bias);
         } else {
-          convert_row<KIND>(r, buf, lane, p);
+          convert_row_transposed<KIND>(r, buf, lane, p);
         }
         ptx::fence_proxy_async_smem();
         __syncwarp();
@@ -686,6 +794,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
     }
     if (lane == 0) ptx::bulk_wait_group_read<0>();  // staging buffers must outlive the stores that read them
+    }
   }
 
   // ------------------------------ teardown ------------------------------
@@ -761,6 +870,8 @@ sp24_status make_im2col_map(CUtensorMap* map, const void* x, int es, uint64_t nb
 
 // 2-D tensor map over a row-major (rows x cols) array of `es`-byte elements with `ld_bytes`
 // between rows; box = box_cols x box_rows elements.
+constexpr int kSwizzle128Atom32 = 1280;
+
 sp24_status encode_map(CUtensorMap* map, const void* base, int es, uint64_t rows, uint64_t cols, uint64_t ld_bytes,
                        uint32_t box_cols, uint32_t box_rows, int swizzle_bytes) {
   EncodeTiledFn fn = encode_fn();
@@ -771,8 +882,11 @@ sp24_status encode_map(CUtensorMap* map, const void* base, int es, uint64_t rows
   cuuint32_t estr[2] = {1, 1};
   CUtensorMapDataType dt = es == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
                                    : (es == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
-  CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
-                                               : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE);
+  // swizzle_bytes: 0, 64, 128, or kSwizzle128Atom32 = the 128-byte pattern in 32-byte units
+  CUtensorMapSwizzle sw = swizzle_bytes == kSwizzle128Atom32
+                              ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B
+                              : (swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                                      : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE));
   CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? SP24_OK : SP24_ERR_CUDA;
@@ -872,7 +986,8 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
     const uint64_t nb = (uint64_t)d->N / ((uint64_t)p.conv_h * p.conv_w);
     st = make_im2col_map(&map_b, B, es, nb, p.conv_h, p.conv_w, p.conv_c, atom_elems, C::kBRows);
   } else if (B_MN) {
-    st = make_map(&map_b, B, es, d->K, d->N, d->ldb * es, C::kBChunkElems, C::kKPerStage, 128);
+    st = make_map(&map_b, B, es, d->K, d->N, d->ldb * es, C::kBChunkElems, C::kKPerStage,
+                  KIND == 2 ? kSwizzle128Atom32 : 128);
   } else {
     st = make_map(&map_b, B, es, d->N, d->K, d->ldb * es, atom_elems, C::kBRows, 128);
   }
@@ -903,7 +1018,12 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
     p.stages = C::kMinStagesFit > C::kMaxStages ? C::kMaxStages : C::kMinStagesFit;
     const int room = C::kSmemLimit - p.stages * C::kStageBytes;
     int epi = 16384;
-    while (epi < 16 * 1024 * cs && 2 * epi <= room) epi *= 2;
+    if (!p.cd_col_major && cs != 1) {
+      // the warps' own loads and stores: one or two 2 KB transposing buffers per epilogue warp
+      if (room >= kEpiWarps * 4096) epi = kEpiWarps * 4096;
+    } else {
+      while (epi < 16 * 1024 * cs && 2 * epi <= room) epi *= 2;
+    }
     p.epi_bytes = epi;
   }
   auto kernel = gemm_kernel<KIND, SPARSE, BLOCK_N, CTAS, MBLK, B_MN>;
@@ -956,8 +1076,7 @@ static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, con
   const bool f8 = is_fp8(d->ab_type);
   const bool fp = d->ab_type == SP24_F16 || d->ab_type == SP24_BF16 || tf32 || f8;
   SP24_RETURN_IF(!fp && d->ab_type != SP24_I8, SP24_ERR_DTYPE);
-  SP24_RETURN_IF(tf32 && (d->cd_type != SP24_F32 || d->order_b != SP24_COL_MAJOR), SP24_ERR_UNSUPPORTED);
-  SP24_RETURN_IF(f8 && d->order_b != SP24_COL_MAJOR, SP24_ERR_UNSUPPORTED);
+  SP24_RETURN_IF(tf32 && d->cd_type != SP24_F32, SP24_ERR_UNSUPPORTED);
   if (dequant)
     SP24_RETURN_IF(fp || (d->cd_type != SP24_BF16 && d->cd_type != SP24_F16 && d->cd_type != SP24_F32 &&
                           d->cd_type != SP24_I8),
@@ -1017,7 +1136,7 @@ struct DequantArgs {
 
 static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A, const void* meta, const void* B,
                             const void* beta, const void* C, void* D, void* workspace, size_t workspace_bytes,
-                            void* stream, const DequantArgs* dq, const ConvArgs* cv = nullptr) {
+                            void* stream, const DequantArgs* dq, const ConvArgs* cv = nullptr, bool acc_f16 = false) {
   bool has_c = false;
   float falpha = 1.f, fbeta = 0.f;
   sp24_status st = validate_gemm(d, alpha, A, meta, B, beta, C, D, workspace, workspace_bytes, has_c, falpha, fbeta,
@@ -1033,6 +1152,7 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
     p.conv_w = (int)cv->w;
     p.conv_c = (int)cv->c;
   }
+  p.acc_f16 = acc_f16 ? 1 : 0;
   if (dq) {
     p.dequant = 1;
     p.relu = dq->relu;
@@ -1075,7 +1195,7 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
     // Few tokens: every n-tile streams all of A again, so the number of n-tiles decides; 256 columns
     // (one accumulator buffer, epilogue not overlapped) when that saves one.  Built for the K-contiguous
     // 16-bit and int8 kinds.
-    const bool has_256 = !tf32 && !f8 && d->order_b == SP24_COL_MAJOR;
+    const bool has_256 = d->order_b == SP24_COL_MAJOR;
     if (has_256 && d->N <= 2048 && (d->N + 255) / 256 < n_tiles) block_n = 256;
   }
   p.band = 16 / mblk;
@@ -1090,7 +1210,7 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
     fprintf(stderr, "sp24_gemm: M=%lld N=%lld K=%lld ab=%d cd=%d %s%s tile=%dx%dx%d band=%d beta=%g%s%s\n", (long long)d->M,
             (long long)d->N, (long long)d->K, (int)d->ab_type, (int)d->cd_type, sparse ? "sparse" : "dense",
             b_mn ? " B:N-contiguous" : "", ctas, block_n, mblk, p.band, (double)fbeta, dq ? " dequant" : "",
-            cv ? " conv3x3" : "");
+            cv ? " conv3x3" : (acc_f16 ? " fp16-accumulate" : ""));
 #define SP24_LAUNCH(K_, BN, CT, MB, MN)                                                               \
   (sparse ? launch<K_, true, BN, CT, MB, MN>(d, p, A, meta, B, s) : launch<K_, false, BN, CT, MB, MN>(d, p, A, meta, B, s))
 #define SP24_DISPATCH(CT, BN, MB)                                                                     \
@@ -1100,7 +1220,9 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
 #define SP24_DISPATCH_F8(CT, BN, MB)                                                                  \
   if (ctas == CT && block_n == BN && mblk == MB && !b_mn && f8) return SP24_LAUNCH(3, BN, CT, MB, false);
 #define SP24_DISPATCH_MN(CT, BN, MB)                                                                  \
-  if (ctas == CT && block_n == BN && mblk == MB && b_mn && !tf32 && !f8) return i8 ? SP24_LAUNCH(1, BN, CT, MB, true) : SP24_LAUNCH(0, BN, CT, MB, true);
+  if (ctas == CT && block_n == BN && mblk == MB && b_mn)                                              \
+    return tf32 ? SP24_LAUNCH(2, BN, CT, MB, true)                                                    \
+                : (f8 ? SP24_LAUNCH(3, BN, CT, MB, true) : (i8 ? SP24_LAUNCH(1, BN, CT, MB, true) : SP24_LAUNCH(0, BN, CT, MB, true)));
   SP24_DISPATCH(1, 128, 1)
   SP24_DISPATCH(2, 224, 1)
   SP24_DISPATCH(2, 224, 2)
@@ -1109,9 +1231,11 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   SP24_DISPATCH_TF32(1, 128, 1)
   SP24_DISPATCH_TF32(2, 224, 1)
   SP24_DISPATCH_TF32(2, 224, 2)
+  SP24_DISPATCH_TF32(2, 256, 1)
   SP24_DISPATCH_F8(1, 128, 1)
   SP24_DISPATCH_F8(2, 224, 1)
   SP24_DISPATCH_F8(2, 224, 2)
+  SP24_DISPATCH_F8(2, 256, 1)
   SP24_DISPATCH_MN(1, 128, 1)
   SP24_DISPATCH_MN(2, 224, 1)
   SP24_DISPATCH_MN(2, 224, 2)
@@ -1127,6 +1251,14 @@ extern "C" sp24_status sp24_gemm(const sp24_gemm_desc* d, const void* alpha, con
                                  const void* B, const void* beta, const void* C, void* D, void* workspace,
                                  size_t workspace_bytes, void* stream) {
   return run_gemm(d, alpha, A, meta, B, beta, C, D, workspace, workspace_bytes, stream, nullptr);
+}
+
+extern "C" sp24_status sp24_gemm_f16acc(const sp24_gemm_desc* d, const void* alpha, const void* A, const void* meta,
+                                        const void* B, const void* beta, const void* C, void* D, void* workspace,
+                                        size_t workspace_bytes, void* stream) {
+  SP24_RETURN_IF(d == nullptr, SP24_ERR_NULL);
+  SP24_RETURN_IF(d->ab_type != SP24_F16 || (d->cd_type != SP24_F16 && d->cd_type != SP24_F32), SP24_ERR_DTYPE);
+  return run_gemm(d, alpha, A, meta, B, beta, C, D, workspace, workspace_bytes, stream, nullptr, nullptr, true);
 }
 
 extern "C" sp24_status sp24_gemm_i8_dequant(const sp24_gemm_desc* d, const void* A, const void* meta, const void* B,

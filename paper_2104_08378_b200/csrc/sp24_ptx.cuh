@@ -151,20 +151,22 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
 }
 
 // ---- descriptors ---------------------------------------------------------------------------------
-// Shared-memory matrix descriptor for a 128-byte-swizzled operand (what the TMA loads write) or,
-// with `swizzle128` false, for 8 x 16-byte core matrices without swizzle.
+// Shared-memory matrix descriptor.  `layout`: kLayoutNone = 8 x 16-byte core matrices without swizzle,
+// kLayoutSw128 = the 128-byte swizzle the TMA loads write, kLayoutSw128Base32 = the 128-byte swizzle
+// in 32-byte units (the only layout of an MN-major tf32 operand).
 //   K-major operand:  rows of 128 bytes along K, 8-row groups `sbo_bytes` (1024) apart; lbo unused.
-//   MN-major operand: rows of 128 bytes along M/N (64 16-bit or 128 8-bit elements), consecutive k
-//                     128 bytes apart, groups of 8 k `sbo_bytes` (1024) apart, 128-byte chunks along
-//                     M/N `lbo_bytes` apart.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t smem_addr, bool swizzle128, uint32_t sbo_bytes,
+//   MN-major operand: rows of 128 bytes along M/N (64 16-bit, 128 8-bit or 32 32-bit elements),
+//                     consecutive k 128 bytes apart, groups of 8 k (4 k for kLayoutSw128Base32)
+//                     `sbo_bytes` apart, 128-byte chunks along M/N `lbo_bytes` apart.
+constexpr uint32_t kLayoutNone = 0, kLayoutSw128Base32 = 1, kLayoutSw128 = 2;
+__device__ __forceinline__ uint64_t smem_desc(uint32_t smem_addr, uint32_t layout, uint32_t sbo_bytes,
                                               uint32_t lbo_bytes = 0) {
   uint64_t d = 0;
   d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
   d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
   d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
   d |= (uint64_t)1 << 46;  // descriptor version for sm_100
-  if (swizzle128) d |= (uint64_t)2 << 61;
+  d |= (uint64_t)layout << 61;
   return d;
 }
 

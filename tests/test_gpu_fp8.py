@@ -100,12 +100,32 @@ def test_fp8_gemm(sp, dtype, dense, shape):
         check_fp(D.to(torch.float64).cpu().numpy(), ref, abs(alpha) * scale, beta_c)
 
 
+@pytest.mark.parametrize("dtype", ["e4m3", "e5m2"])
+@pytest.mark.parametrize("dense", [False, True])
+@pytest.mark.parametrize("shape", [(128, 128, 128), (160, 288, 416), (512, 1344, 1024)])
+def test_fp8_b_stored_n_contiguous(sp, dtype, dense, shape):
+    """order_b = ROW_MAJOR for the 8-bit floats: the K x N matrix stored row by row (MN-major operand)."""
+    M, N, K = shape
+    A = _rand(M, K, dtype, 17)
+    Bt = _rand(N, K, dtype, 18, ("uniform", -1.0, 1.0), tensor=6)
+    v_ref, m_ref, _ = oracle.compress(A, dtype)
+    Ad = _dev(A, dtype)
+    Bkn = _dev(np.ascontiguousarray(Bt.T), dtype)                 # [K, N], N contiguous
+    if dense:
+        D = sp.gemm(sp.prune(Ad), None, Bkn, cd="f32", a_is_dense=True, b_row_major=True)
+    else:
+        vals, meta, _ = sp.compress(Ad, layout=sp.META_TCGEN05)
+        D = sp.gemm(vals, meta, Bkn, cd="f32", b_row_major=True)
+    torch.cuda.synchronize()
+    assert sp.gemm_status(device=D.device) == 0
+    ref = oracle.gemm_sparse(v_ref, m_ref, Bt, dtype)
+    check_fp(D.to(torch.float64).cpu().numpy(), ref, oracle.gemm_abs(v_ref, m_ref, Bt, dtype))
+
+
 def test_fp8_rejections(sp):
     A = torch.zeros(128, 64, dtype=torch.uint8, device="cuda").view(torch.float8_e4m3fn)
     Bt = torch.zeros(128, 128, dtype=torch.uint8, device="cuda").view(torch.float8_e4m3fn)
     meta = torch.zeros(4096, dtype=torch.uint8, device="cuda")
-    with pytest.raises(RuntimeError):      # N-contiguous B is not built for the 8-bit floats
-        sp.gemm(A, meta, Bt, b_row_major=True)
     with pytest.raises(RuntimeError):      # the accumulator is fp32: no integer output
         sp.gemm(A, meta, Bt, cd="i32")
     with pytest.raises(RuntimeError):      # magnitude sums are defined for the paper's types only

@@ -70,6 +70,26 @@ def test_tf32_gemm(sp, dense, shape):
         check_fp(got, ref, abs(alpha) * mag, beta_c)
 
 
+@pytest.mark.parametrize("dense", [False, True])
+@pytest.mark.parametrize("shape", [(128, 128, 64), (144, 272, 208), (512, 1344, 512)])
+def test_tf32_b_stored_n_contiguous(sp, dense, shape):
+    """order_b = ROW_MAJOR in the TF32 mode: the K x N matrix stored row by row (MN-major operand, which for
+    32-bit elements exists only in the 128-byte swizzle with 32-byte units)."""
+    M, N, K = shape
+    A, Bt = _rand(M, K, 27), _rand(N, K, 28, ("uniform", -1.0, 1.0))
+    v_ref, m_ref, _ = oracle.compress_1of2(A)
+    Ad, Bkn = _dev(A), _dev(np.ascontiguousarray(Bt.T))          # [K, N], N contiguous
+    if dense:
+        D = sp.gemm(sp.prune(Ad), None, Bkn, a_is_dense=True, b_row_major=True)
+    else:
+        vals, meta, _ = sp.compress(Ad)
+        D = sp.gemm(vals, meta, Bkn, b_row_major=True)
+    torch.cuda.synchronize()
+    assert sp.gemm_status(device=D.device) == 0
+    ref, mag = oracle.gemm_sparse_1of2(v_ref, m_ref, Bt)
+    check_fp(D.double().cpu().numpy(), ref, mag)
+
+
 def test_tf32_identity_b_is_exact(sp):
     M, K = 256, 192
     A = _rand(M, K, 11)

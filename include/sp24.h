@@ -173,6 +173,11 @@ typedef struct {
   int a_is_dense;
 } sp24_gemm_desc;
 
+/* Reports the tile shape sp24_gemm (and its variants) would use for this problem on the current
+ * device: CTAs per tile (1, or 2 = a pair working on one tile), columns per tile, 128-row blocks
+ * per CTA.  The output tile is (128 * ctas * mblk) x block_n.  Launches nothing. */
+sp24_status sp24_gemm_plan(const sp24_gemm_desc* d, int* ctas, int* block_n, int* mblk);
+
 /* Bytes of device workspace sp24_gemm needs for this problem (currently a fixed 256 bytes:
  * the device-side status record).  The workspace must be 16-byte aligned. */
 size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d);

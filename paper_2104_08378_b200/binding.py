@@ -33,6 +33,7 @@ EXPORTS = [
     "sp24_im2col_nhwc_3x3", "sp24_pipeline_host", "sp24_gemm_static_ws", "sp24_gemm_i8_dequant",
     "sp24_conv3x3_nhwc", "sp24_kept_magnitude", "sp24_apply_mask", "sp24_prune_2d",
     "sp24_gemm_static_ws_status", "sp24_set_tile_override", "sp24_test_set_fault_hooks", "sp24_gemm_f16acc",
+    "sp24_gemm_plan",
 ]
 
 
@@ -70,6 +71,8 @@ def _load() -> ctypes.CDLL:
     lib.sp24_gemm_workspace_bytes.argtypes = [ctypes.POINTER(GemmDesc)]
     lib.sp24_gemm_workspace_bytes.restype = sz
     lib.sp24_gemm.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sp24_gemm_plan.argtypes = [ctypes.POINTER(GemmDesc), ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)]
+    lib.sp24_gemm_plan.restype = ci
     lib.sp24_gemm_f16acc.argtypes = lib.sp24_gemm.argtypes
     lib.sp24_gemm_f16acc.restype = ci
     lib.sp24_gemm_static_ws.argtypes = [ctypes.POINTER(GemmDesc), vp, vp, vp, vp, vp, vp, vp, vp]
@@ -239,6 +242,13 @@ def gemm(A: torch.Tensor, meta: torch.Tensor | None, Bt: torch.Tensor, *, alpha=
               ctypes.byref(b), _ptr(C), _ptr(out), _ptr(ws), ws.numel(), _stream()),
            "sp24_gemm_f16acc" if acc_f16 else "sp24_gemm")
     return out
+
+
+def gemm_plan(desc: GemmDesc) -> str:
+    """sp24_gemm_plan: the tile shape the library picks for this problem, as "<ctas>x<block_n>x<mblk>"."""
+    c, n, m = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    _check(lib.sp24_gemm_plan(ctypes.byref(desc), ctypes.byref(c), ctypes.byref(n), ctypes.byref(m)), "sp24_gemm_plan")
+    return f"{c.value}x{n.value}x{m.value}"
 
 
 def gemm_status(ws: torch.Tensor | None = None, device=None) -> int:

@@ -111,7 +111,9 @@ struct Cfg {
   static constexpr int kMmasPerStage = SPARSE ? 4 : 4 * kBBoxes;   // per m-block
   static constexpr int kSmemBytes = 232448;  // always the whole opt-in maximum
   static_assert(kMinStagesFit >= 2, "need at least two stages");
-  static_assert(BLOCK_N % 32 == 0, "the epilogue moves 32-column boxes");
+  // the epilogue moves 32-column boxes; a last box of 16 columns (240-column tiles) is handled only by
+  // the epilogue for row-major outputs, which bounds every access by the tile's last column
+  static_assert(BLOCK_N % 16 == 0, "tile width");
   static_assert(kStageBytes % 1024 == 0, "stages must keep the 1024-byte alignment of the atoms");
   static_assert(kECol + (SPARSE ? 2 * MBLK * 8 : 0) <= (int)kTmemCols, "tensor memory overflow");
 };
@@ -335,7 +337,7 @@ template <int KIND, int CS, int BLOCK_N, int CTAS, int MBLK, int ACC_STAGES>
 __device__ __forceinline__ void epilogue_rows(const GemmParams& p, Shared* sh, uint8_t* epi, uint32_t tmem_base,
                                               int cta_rank, int cluster_id, int num_clusters, int num_tiles, int warp,
                                               int lane) {
-  constexpr int kSub = BLOCK_N / 32, kIters = MBLK * kSub;
+  constexpr int kSub = (BLOCK_N + 31) / 32, kIters = MBLK * kSub;  // the last box of a 240-column tile is half a box
   constexpr int kBoxes = (kIters + 1) / 2;  // boxes per warp and tile (the two warps of a lane quarter alternate)
   constexpr int W = 8 * CS;                 // 32-bit words of one box row
   constexpr int P = CS == 2 ? 4 : 1;        // boxes whose C values are held in registers
@@ -355,6 +357,7 @@ __device__ __forceinline__ void epilogue_rows(const GemmParams& p, Shared* sh, u
   for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
     int mt, nt;
     tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
+    const int col_end = min(N, (nt + 1) * BLOCK_N);  // columns of this tile stop here
     // box n of this warp in this tile: first row / column, accumulator column, inside the matrix?
     auto geom = [&](int n, int& row0, int& col0, int& tcol) -> bool {
       const int it = half + 2 * n;
@@ -362,7 +365,7 @@ __device__ __forceinline__ void epilogue_rows(const GemmParams& p, Shared* sh, u
       row0 = ((mt * MBLK + j) * CTAS + cta_rank) * kBlockM + q * 32;
       col0 = nt * BLOCK_N + sc * 32;
       tcol = j * BLOCK_N + sc * 32;
-      return it < kIters && row0 < M && col0 < N;
+      return it < kIters && row0 < M && col0 < col_end;
     };
     auto load_c = [&](int n, uint32_t (&c)[W]) {
       int row0, col0, tcol;
@@ -372,7 +375,7 @@ __device__ __forceinline__ void epilogue_rows(const GemmParams& p, Shared* sh, u
       const uint4* src = reinterpret_cast<const uint4*>(Cb + (size_t)row * ldc_b + (size_t)col0 * CS);
 #pragma unroll
       for (int v = 0; v < W / 4; ++v) {
-        if (col0 + v * kUnitElems < N) {
+        if (col0 + v * kUnitElems < col_end) {
           const uint4 x = src[v];
           c[4 * v] = x.x; c[4 * v + 1] = x.y; c[4 * v + 2] = x.z; c[4 * v + 3] = x.w;
         }
@@ -440,7 +443,7 @@ __device__ __forceinline__ void epilogue_rows(const GemmParams& p, Shared* sh, u
             const int i = lane + 32 * k, rr = i >> 2, u = i & 3;
             const uint4 x = *reinterpret_cast<const uint4*>(buf + rr * 64 + ((u ^ ((rr >> 1) & 3)) << 4));
             const int grow = row0 + rr, gcol = col0 + ps * (64 / CS) + u * kUnitElems;
-            if (grow < M && gcol < N) *reinterpret_cast<uint4*>(Db + (size_t)grow * ldd_b + (size_t)gcol * CS) = x;
+            if (grow < M && gcol < col_end) *reinterpret_cast<uint4*>(Db + (size_t)grow * ldd_b + (size_t)gcol * CS) = x;
           }
           ++pass_no;
         }
@@ -1068,6 +1071,46 @@ extern "C" size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d) {
   return 256;
 }
 
+// Tile choice.  Large problems (at least six waves of tiles): a pair of CTAs with two m-blocks each,
+// 512 x 224 tiles: least operand traffic per flop.  Medium: a pair with one m-block and two
+// accumulator buffers (epilogue overlapped), 256 x 224 -- or 256 x 240 where that takes the pairs
+// one round of tiles fewer (224: two fp32 accumulators plus the metadata columns fit the 512 columns
+// of tensor memory and 224 is a multiple of 32; 240 is the widest multiple of 16 that fits, built for
+// the 16-bit kinds with K-contiguous B and row-major output).  Small: single CTAs, 128 x 128.
+static void choose_tile(const sp24_gemm_desc* d, int& ctas, int& block_n, int& mblk) {
+  const int64_t n224 = (d->N + 223) / 224;
+  ctas = 1; block_n = 128; mblk = 1;
+  if (d->M >= 512 && (d->M / 512) * n224 >= 444) {
+    ctas = 2; block_n = 224; mblk = 2;
+    return;
+  }
+  if (d->M >= 256 && (d->M / 256) * n224 >= 32) {
+    ctas = 2; block_n = 224; mblk = 1;
+    const int64_t m_tiles = (d->M + 255) / 256, pairs = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
+    const bool has_240 = (d->ab_type == SP24_F16 || d->ab_type == SP24_BF16) && d->order_b == SP24_COL_MAJOR &&
+                         d->order_d == SP24_ROW_MAJOR;
+    const int64_t rounds224 = (m_tiles * n224 + pairs - 1) / pairs;
+    const int64_t rounds240 = (m_tiles * ((d->N + 239) / 240) + pairs - 1) / pairs;
+    if (has_240 && rounds240 < rounds224) block_n = 240;
+    // Few tokens: every n-tile streams all of A again, so the number of n-tiles decides; 256 columns
+    // (one accumulator buffer, epilogue not overlapped) when that saves one.  Built for K-contiguous B.
+    if (d->order_b == SP24_COL_MAJOR && d->N <= 2048 && (d->N + 255) / 256 < (d->N + block_n - 1) / block_n) block_n = 256;
+  }
+}
+
+extern "C" sp24_status sp24_gemm_plan(const sp24_gemm_desc* d, int* ctas, int* block_n, int* mblk) {
+  SP24_RETURN_IF(d == nullptr || ctas == nullptr || block_n == nullptr || mblk == nullptr, SP24_ERR_NULL);
+  SP24_RETURN_IF(d->M <= 0 || d->N <= 0 || d->K <= 0, SP24_ERR_SHAPE);
+  choose_tile(d, *ctas, *block_n, *mblk);
+  Settings& cfg = settings();
+  if (const int c = cfg.ctas.load(std::memory_order_relaxed)) {
+    *ctas = c;
+    *block_n = cfg.block_n.load(std::memory_order_relaxed);
+    *mblk = cfg.mblk.load(std::memory_order_relaxed);
+  }
+  return SP24_OK;
+}
+
 static sp24_status validate_gemm(const sp24_gemm_desc* d, const void* alpha, const void* A, const void* meta,
                                  const void* B, const void* beta, const void* C, void* D, void* ws, size_t ws_bytes,
                                  bool& has_c, float& falpha, float& fbeta, bool dequant = false) {
@@ -1182,22 +1225,8 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   p.cd_col_major = d->order_d == SP24_COL_MAJOR ? 1 : 0;
   const bool sparse = !d->a_is_dense;
   const bool i8 = d->ab_type == SP24_I8, tf32 = d->ab_type == SP24_F32, f8 = is_fp8(d->ab_type);
-  // Tile choice.  Large problems (at least six waves of tiles): a pair of CTAs with two m-blocks
-  // each, 512 x 224 tiles: least operand traffic per flop.  Medium: a pair with one m-block, 256 x 224,
-  // epilogue overlapped.  Small: single CTAs, 128 x 128.  (224: two fp32 accumulators plus the
-  // metadata columns fit the 512 columns of tensor memory, and 224 is a multiple of 32.)
-  // SP24_TILE=<ctas>x<block_n>x<mblk> overrides (benchmarking).
-  const int64_t n_tiles = (d->N + 223) / 224;
-  int ctas = 1, block_n = 128, mblk = 1;
-  if (d->M >= 512 && (d->M / 512) * n_tiles >= 444) { ctas = 2; block_n = 224; mblk = 2; }
-  else if (d->M >= 256 && (d->M / 256) * n_tiles >= 32) {
-    ctas = 2; block_n = 224; mblk = 1;
-    // Few tokens: every n-tile streams all of A again, so the number of n-tiles decides; 256 columns
-    // (one accumulator buffer, epilogue not overlapped) when that saves one.  Built for the K-contiguous
-    // 16-bit and int8 kinds.
-    const bool has_256 = d->order_b == SP24_COL_MAJOR;
-    if (has_256 && d->N <= 2048 && (d->N + 255) / 256 < n_tiles) block_n = 256;
-  }
+  int ctas, block_n, mblk;
+  choose_tile(d, ctas, block_n, mblk);
   p.band = 16 / mblk;
   if (const int c = cfg.ctas.load(std::memory_order_relaxed)) {
     ctas = c;
@@ -1228,6 +1257,8 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   SP24_DISPATCH(2, 224, 2)
   SP24_DISPATCH(2, 192, 2)
   SP24_DISPATCH(2, 256, 1)
+  if (ctas == 2 && block_n == 240 && mblk == 1 && !b_mn && !tf32 && !f8 && !i8 && !p.cd_col_major && elem_bytes(d->cd_type) != 1)
+    return SP24_LAUNCH(0, 240, 2, 1, false);
   SP24_DISPATCH_TF32(1, 128, 1)
   SP24_DISPATCH_TF32(2, 224, 1)
   SP24_DISPATCH_TF32(2, 224, 2)

@@ -69,8 +69,10 @@ def test_streaming_kernels_stay_inside_their_outputs(sp, dtype, shape):
 
 
 @pytest.mark.parametrize("kind", ["bf16", "i8", "e4m3", "tf32"])
-@pytest.mark.parametrize("tile", ["1x128x1", "2x224x1", "2x224x2"])
+@pytest.mark.parametrize("tile", ["1x128x1", "2x224x1", "2x224x2", "2x240x1"])
 def test_gemm_stays_inside_d(sp, force_tile, kind, tile):
+    if tile == "2x240x1" and kind != "bf16":
+        pytest.skip("240-column tiles are built for the 16-bit kinds")
     M, N, K = 1184, 736, 640
     if kind == "i8":
         A = torch.randint(-127, 128, (M, K), dtype=torch.int8, device="cuda")
@@ -92,7 +94,7 @@ def test_gemm_stays_inside_d(sp, force_tile, kind, tile):
         torch.cuda.synchronize()
         assert sp.gemm_status(ws) == 0
         D.check(f"gemm {kind} {tile}")
-    if kind in ("bf16", "i8"):
+    if kind in ("bf16", "i8") and tile != "2x240x1":   # (240 columns: row-major outputs only)
         Dt = Guarded(N, M, cdt, M + 32)              # column-major D (M contiguous)
         sp.gemm(vals, meta, Bt, out=Dt.t, cd=cd, cd_col_major=True, ws=ws)
         torch.cuda.synchronize()

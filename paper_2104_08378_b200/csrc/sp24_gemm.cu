@@ -40,7 +40,11 @@ namespace {
 constexpr int kBlockM = 128;              // rows of A per CTA and m-block (tensor-memory lanes)
 constexpr int kAtomBytes = 128;           // bytes per row of one swizzle-128B operand atom
 constexpr int kEpiWarps = 8;              // two per tensor-memory lane quarter, taking alternate boxes
-constexpr int kNumThreads = 64 + 32 * kEpiWarps;  // TMA producer, MMA issuer, epilogue warps
+constexpr int kFirstEpiWarp = 2;          // warp 0: TMA producer, warp 1: MMA issuer
+constexpr int kNumThreads = 32 * (kFirstEpiWarp + kEpiWarps);
+// (Ten warps leave three on two of the SM's four sub-partitions, which caps the kernel at 168
+// registers per thread; trading registers between the roles with setmaxnreg was tried and made the
+// compiler spill far more than it saved.)
 constexpr long long kWaitTimeoutCycles = 2000ll * 1000ll * 1000ll;  // per wait: 1-2 s of SM clock
 constexpr uint32_t kTmemCols = 512;
 
@@ -343,7 +347,7 @@ __device__ __forceinline__ void epilogue_rows(const GemmParams& p, Shared* sh, u
   constexpr int P = CS == 2 ? 4 : 1;        // boxes whose C values are held in registers
   constexpr int kPasses = CS / 2;
   constexpr int kUnitElems = 16 / CS;       // elements per 16-byte unit
-  const int q = warp & 3, ew = warp - 2, half = ew >> 2;
+  const int q = warp & 3, ew = warp - kFirstEpiWarp, half = ew >> 2;
   const int nbuf = p.epi_bytes >= kEpiWarps * 4096 ? 2 : 1;
   uint8_t* stage = epi + ew * (nbuf * 2048);
   const uint8_t* Cb = static_cast<const uint8_t*>(p.C);
@@ -446,6 +450,161 @@ __device__ __forceinline__ void epilogue_rows(const GemmParams& p, Shared* sh, u
             if (grow < M && gcol < col_end) *reinterpret_cast<uint4*>(Db + (size_t)grow * ldd_b + (size_t)gcol * CS) = x;
           }
           ++pass_no;
+        }
+      }
+    }
+    if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+  }
+}
+
+// The same epilogue in chunks of 128 bytes per row (64 columns of a 2-byte type = two boxes, 32
+// columns of a 4-byte type), used when every epilogue warp can have a 4 KB buffer.  Whole 128-byte
+// lines per request matter: what the L2 serves per unit of time is requests more than bytes, and a
+// C load of 16 bytes per row (a thread fetching its own accumulator row) costs the GEMM about 10 %.
+// So C is loaded the way D is stored -- eight lanes per row, four rows per instruction -- into
+// registers, ahead of time, and reaches the thread that owns the row through the warp's buffer:
+// C chunk -> buffer, each thread converts ITS row in place, buffer -> D.
+template <int KIND, int CS, int BLOCK_N, int CTAS, int MBLK, int ACC_STAGES>
+__device__ __forceinline__ void epilogue_rows_wide(const GemmParams& p, Shared* sh, uint8_t* epi, uint32_t tmem_base,
+                                                   int cta_rank, int cluster_id, int num_clusters, int num_tiles,
+                                                   int warp, int lane) {
+  constexpr int kSub = (BLOCK_N + 31) / 32;                 // boxes per m-block (the last one may be half a box)
+  constexpr int kChunkBoxes = 4 / CS;                       // boxes per chunk: 2 (2-byte types) or 1
+  constexpr int kChunkCols = 128 / CS;
+  constexpr int kChunksPerBlock = (kSub + kChunkBoxes - 1) / kChunkBoxes;
+  // two m-blocks: the two warps of a lane quarter take one m-block each; one m-block: alternate chunks
+  constexpr int kMyChunks = MBLK == 2 ? kChunksPerBlock : (kChunksPerBlock + 1) / 2;
+  constexpr int kMyBoxes = kMyChunks * kChunkBoxes;
+  constexpr int W = 8 * CS;                                 // 32-bit words of one box row
+  constexpr int kBoxUnits = 2 * CS;                         // 16-byte units of one box row
+  constexpr int P = CS == 2 ? 2 : 1;                        // chunks whose C values are held in registers (32 each)
+  constexpr int kUnitElems = 16 / CS;
+  const int q = warp & 3, ew = warp - kFirstEpiWarp, half = ew >> 2;
+  uint8_t* buf = epi + ew * 4096;
+  const uint8_t* Cb = static_cast<const uint8_t*>(p.C);
+  uint8_t* Db = static_cast<uint8_t*>(p.D);
+  const size_t ldc_b = (size_t)p.ldc * CS, ldd_b = (size_t)p.ldd * CS;
+  const int M = (int)p.M, N = (int)p.N;
+  const bool has_c = p.has_c != 0;
+  uint4 creg[P][8];
+  int acc = 0;
+  uint32_t acc_phase = 0;
+  // chunk n of this warp: m-block and chunk column inside the tile
+  auto chunk_of = [&](int n, int& j, int& c) -> bool {
+    j = MBLK == 2 ? half : 0;
+    c = MBLK == 2 ? n : half + 2 * n;
+    return c < kChunksPerBlock;
+  };
+  // box m of this warp (box m % kChunkBoxes of chunk m / kChunkBoxes): accumulator column; does it exist?
+  auto box_of = [&](int m, int& tcol) -> bool {
+    int j, c;
+    const bool ok = chunk_of(m / kChunkBoxes, j, c);
+    const int sc = c * kChunkBoxes + m % kChunkBoxes;
+    tcol = j * BLOCK_N + sc * 32;
+    return ok && sc < kSub;
+  };
+  for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
+    int mt, nt;
+    tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
+    const int col_end = min(N, (nt + 1) * BLOCK_N);  // columns of this tile stop here
+    auto geom = [&](int n, int& row0, int& col0) -> bool {
+      int j, c;
+      const bool ok = chunk_of(n, j, c);
+      row0 = ((mt * MBLK + j) * CTAS + cta_rank) * kBlockM + q * 32;
+      col0 = nt * BLOCK_N + c * kChunkCols;
+      return ok && row0 < M && col0 < col_end;
+    };
+    auto load_c = [&](int n, uint4 (&c)[8]) {
+      int row0, col0;
+      if (!geom(n, row0, col0)) return;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int i = lane + 32 * k, rr = i >> 3, u = i & 7;
+        const int grow = row0 + rr, gcol = col0 + u * kUnitElems;
+        if (grow < M && gcol < col_end) c[k] = *reinterpret_cast<const uint4*>(Cb + (size_t)grow * ldc_b + (size_t)gcol * CS);
+      }
+    };
+    if (has_c) {
+#pragma unroll
+      for (int n = 0; n < P; ++n)
+        if (n < kMyChunks) load_c(n, creg[n]);
+    }
+    if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u, p.wait_limit)) break;
+    ptx::tc_fence_after();
+    const uint32_t t_acc = tmem_base + (acc * MBLK) * BLOCK_N + ((uint32_t)(q * 32) << 16);
+    uint32_t racc[2][32];
+    {
+      int tcol;
+      box_of(0, tcol);  // every warp has at least one box
+      ptx::tmem_ld_32x32b_x32(t_acc + tcol, racc[0]);
+    }
+#pragma unroll
+    for (int n = 0; n < kMyChunks; ++n) {
+      int row0, col0;
+      const bool live = geom(n, row0, col0);  // same answer for the whole warp
+      __syncwarp();  // the reads of the previous chunk's store phase are done
+      if (has_c) {
+        if (live) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const int i = lane + 32 * k, rr = i >> 3, u = i & 7;
+            *reinterpret_cast<uint4*>(buf + rr * 128 + ((u ^ (rr & 7)) << 4)) = creg[n % P][k];
+          }
+        }
+        // the C registers of chunk n are free: fetch chunk n + P into them
+        if (n + P < kMyChunks) load_c(n + P, creg[n % P]);
+        __syncwarp();
+      }
+#pragma unroll
+      for (int b = 0; b < kChunkBoxes; ++b) {
+        const int m = n * kChunkBoxes + b;
+        int tcol;
+        if (!box_of(m, tcol)) break;  // same answer for the whole warp; boxes that exist form a prefix
+        ptx::tmem_ld_wait();
+        int tcol1;
+        if (m + 1 < kMyBoxes && box_of(m + 1, tcol1)) {
+          ptx::tmem_ld_32x32b_x32(t_acc + tcol1, racc[(m + 1) & 1]);
+        } else {
+          // this warp's part of the accumulators is in registers: hand it back to the MMA issuer (CTA 0 of the pair)
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            if (CTAS == 1) ptx::mbar_arrive(&sh->tmem_empty[acc]);
+            else ptx::mbar_arrive_cluster(&sh->tmem_empty[acc], 0);
+          }
+        }
+        if (!live) continue;
+        uint32_t (&r)[32] = racc[m & 1];
+        if (KIND == 0 && p.acc_f16) widen_f16_accumulators(r);
+        float scale = 1.f, bias = 0.f;
+        if (KIND == 1 && p.dequant) {
+          const int row = min(row0 + lane, M - 1);
+          scale = __ldg(p.row_scale + row);
+          bias = p.bias ? __ldg(p.bias + row) : 0.f;
+        }
+        uint32_t c[W], o[W];
+        uint8_t* my_row = buf + lane * 128;
+        if (has_c) {
+#pragma unroll
+          for (int v = 0; v < kBoxUnits; ++v) {
+            const uint4 x = *reinterpret_cast<const uint4*>(my_row + (((b * kBoxUnits + v) ^ (lane & 7)) << 4));
+            c[4 * v] = x.x; c[4 * v + 1] = x.y; c[4 * v + 2] = x.z; c[4 * v + 3] = x.w;
+          }
+        }
+        compute_row<KIND, CS>(r, c, has_c, p, scale, bias, o);
+#pragma unroll
+        for (int v = 0; v < kBoxUnits; ++v)
+          *reinterpret_cast<uint4*>(my_row + (((b * kBoxUnits + v) ^ (lane & 7)) << 4)) =
+              make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+      }
+      if (live) {
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int i = lane + 32 * k, rr = i >> 3, u = i & 7;
+          const uint4 x = *reinterpret_cast<const uint4*>(buf + rr * 128 + ((u ^ (rr & 7)) << 4));
+          const int grow = row0 + rr, gcol = col0 + u * kUnitElems;
+          if (grow < M && gcol < col_end) *reinterpret_cast<uint4*>(Db + (size_t)grow * ldd_b + (size_t)gcol * CS) = x;
         }
       }
     }
@@ -663,24 +822,29 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
       }
     }
-  } else {
+  } else if (warp >= kFirstEpiWarp) {
     // ------------------------------ epilogue ------------------------------
     const int cs = elem_bytes((sp24_dtype)p.cd_type);
     if (!p.cd_col_major && cs != 1) {
-      // row-major C / D: loads and stores by the epilogue warps themselves
-      if (KIND != 2 && cs == 2)
-        epilogue_rows<KIND, 2, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id,
-                                                                   num_clusters, num_tiles, warp, lane);
-      else
-        epilogue_rows<KIND, 4, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id,
-                                                                   num_clusters, num_tiles, warp, lane);
+      // row-major C / D: loads and stores by the epilogue warps themselves.  With C (beta != 0) in 128-byte
+      // chunks per row, if each warp can have a 4 KB buffer: the coalesced C loads are worth 8 % of the
+      // large bf16 GEMM.  Without C in 64-byte passes through two 2 KB buffers, which is the faster
+      // form for the stores alone (int8 4096 x 8192 x 4096: 80 against 88 us).
+      const bool wide = p.has_c && p.epi_bytes >= kEpiWarps * 4096;
+      if (KIND != 2 && cs == 2) {
+        if (wide) epilogue_rows_wide<KIND, 2, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id, num_clusters, num_tiles, warp, lane);
+        else epilogue_rows<KIND, 2, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id, num_clusters, num_tiles, warp, lane);
+      } else {
+        if (wide) epilogue_rows_wide<KIND, 4, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id, num_clusters, num_tiles, warp, lane);
+        else epilogue_rows<KIND, 4, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id, num_clusters, num_tiles, warp, lane);
+      }
     } else {
     // Column-major C / D and 1-byte outputs.  Each warp owns 32 accumulator rows and walks its tiles in
     // 32 x 32 boxes: TMA load of the C box (if beta != 0) into a staging buffer a few boxes ahead,
     // tcgen05.ld of the accumulator columns, convert in place, TMA store of the D box.  Boxes outside
     // the matrix are clipped by the TMA.
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
-    const int ew = warp - 2;  // epilogue warp 0..7: warps ew and ew + 4 share a lane quarter
+    const int ew = warp - kFirstEpiWarp;  // epilogue warp 0..7: warps ew and ew + 4 share a lane quarter
     const int buf_bytes = 1024 * cs;
     // Both warps of a quarter work (alternate boxes) when each can have a staging buffer of its own;
     // otherwise the second one only takes part in handing the accumulators back.

@@ -10,8 +10,11 @@
 //            back to the producer and, after the last k-block, the accumulators to the epilogue;
 //            owns the tensor-memory allocation;
 //   warps 2-9 epilogue, two per tensor-memory lane quarter taking alternate 32-column boxes:
-//            tcgen05.ld accumulator -> registers, alpha/beta, convert into a staging buffer, TMA
-//            store; the TMA loads of C run a few boxes ahead, the next tcgen05.ld one box ahead.
+//            tcgen05.ld accumulator -> registers (the next box's load already under way), alpha /
+//            beta / conversion in registers, then one of two forms.  Row-major 2-byte outputs: the
+//            warps load C and store D themselves, through small per-warp transposing buffers, and
+//            hand the accumulators back as soon as their last box is in registers.  Other outputs:
+//            a staging box per warp, C boxes TMA-loaded a few boxes ahead, TMA store of the D box.
 // CTAS == 2 runs a pair of CTAs (cluster of two): each CTA loads its 128 rows of A / metadata per
 // m-block and its half of B, CTA 0 issues cta_group::2 MMAs (M = 256) for both.
 // MBLK == 2 gives every CTA two m-blocks (two accumulators, one B tile): what an SM can pull in
@@ -61,6 +64,7 @@ struct GemmParams {
   int32_t cd_type;    // sp24_dtype of C / D
   int32_t has_c;
   int32_t stages, epi_bytes;  // shared memory: ring stages and bytes of epilogue staging
+  int32_t epi_lsu;            // epilogue form: 1 = the warps' own loads and stores, 0 = TMA through staging boxes
   long long wait_limit;       // SM cycles after which a device-side wait gives up
   int32_t test_skip_stage;    // test hook: the producers leave out one k-block, so that a wait expires
   int32_t band;       // m-tiles per band of the tile sweep
@@ -252,6 +256,27 @@ __device__ __forceinline__ void widen_f16_accumulators(uint32_t (&r)[32]) {
   for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__half2float(__ushort_as_half((unsigned short)(r[e] & 0xFFFFu))));
 }
 
+// TMA-staged form of a 4-byte row-major box (rows of 128 bytes in the TMA's 128-byte swizzle: 16-byte
+// unit v of row r sits at unit v ^ (r & 7), which also keeps the row-per-thread accesses free of bank
+// conflicts): C, if any, is in the staging buffer; the result replaces it there.
+template <int KIND>
+__device__ __forceinline__ void convert_row_staged(const uint32_t (&r)[32], uint8_t* buf, int lane, const GemmParams& p,
+                                                   float scale, float bias) {
+  uint32_t c[32], o[32];
+  uint8_t* row = buf + lane * 128;
+  if (p.has_c) {
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+      const uint4 x = *reinterpret_cast<const uint4*>(row + ((v ^ (lane & 7)) << 4));
+      c[4 * v] = x.x; c[4 * v + 1] = x.y; c[4 * v + 2] = x.z; c[4 * v + 3] = x.w;
+    }
+  }
+  compute_row<KIND, 4>(r, c, p.has_c != 0, p, scale, bias, o);
+#pragma unroll
+  for (int v = 0; v < 8; ++v)
+    *reinterpret_cast<uint4*>(row + ((v ^ (lane & 7)) << 4)) = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+}
+
 // int8 output of the dequantising epilogue: rows of 32 bytes, no swizzle
 __device__ __forceinline__ void convert_row_dequant_i8(const uint32_t (&r)[32], uint8_t* buf, int lane, const GemmParams& p,
                                                        float scale, float bias) {
@@ -344,7 +369,7 @@ __device__ __forceinline__ void epilogue_rows(const GemmParams& p, Shared* sh, u
   constexpr int kSub = (BLOCK_N + 31) / 32, kIters = MBLK * kSub;  // the last box of a 240-column tile is half a box
   constexpr int kBoxes = (kIters + 1) / 2;  // boxes per warp and tile (the two warps of a lane quarter alternate)
   constexpr int W = 8 * CS;                 // 32-bit words of one box row
-  constexpr int P = CS == 2 ? 4 : 1;        // boxes whose C values are held in registers
+  constexpr int P = CS == 2 ? 4 : 1;        // boxes whose C values are held in registers (16 or 32 registers each)
   constexpr int kPasses = CS / 2;
   constexpr int kUnitElems = 16 / CS;       // elements per 16-byte unit
   const int q = warp & 3, ew = warp - kFirstEpiWarp, half = ew >> 2;
@@ -450,161 +475,6 @@ __device__ __forceinline__ void epilogue_rows(const GemmParams& p, Shared* sh, u
             if (grow < M && gcol < col_end) *reinterpret_cast<uint4*>(Db + (size_t)grow * ldd_b + (size_t)gcol * CS) = x;
           }
           ++pass_no;
-        }
-      }
-    }
-    if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
-  }
-}
-
-// The same epilogue in chunks of 128 bytes per row (64 columns of a 2-byte type = two boxes, 32
-// columns of a 4-byte type), used when every epilogue warp can have a 4 KB buffer.  Whole 128-byte
-// lines per request matter: what the L2 serves per unit of time is requests more than bytes, and a
-// C load of 16 bytes per row (a thread fetching its own accumulator row) costs the GEMM about 10 %.
-// So C is loaded the way D is stored -- eight lanes per row, four rows per instruction -- into
-// registers, ahead of time, and reaches the thread that owns the row through the warp's buffer:
-// C chunk -> buffer, each thread converts ITS row in place, buffer -> D.
-template <int KIND, int CS, int BLOCK_N, int CTAS, int MBLK, int ACC_STAGES>
-__device__ __forceinline__ void epilogue_rows_wide(const GemmParams& p, Shared* sh, uint8_t* epi, uint32_t tmem_base,
-                                                   int cta_rank, int cluster_id, int num_clusters, int num_tiles,
-                                                   int warp, int lane) {
-  constexpr int kSub = (BLOCK_N + 31) / 32;                 // boxes per m-block (the last one may be half a box)
-  constexpr int kChunkBoxes = 4 / CS;                       // boxes per chunk: 2 (2-byte types) or 1
-  constexpr int kChunkCols = 128 / CS;
-  constexpr int kChunksPerBlock = (kSub + kChunkBoxes - 1) / kChunkBoxes;
-  // two m-blocks: the two warps of a lane quarter take one m-block each; one m-block: alternate chunks
-  constexpr int kMyChunks = MBLK == 2 ? kChunksPerBlock : (kChunksPerBlock + 1) / 2;
-  constexpr int kMyBoxes = kMyChunks * kChunkBoxes;
-  constexpr int W = 8 * CS;                                 // 32-bit words of one box row
-  constexpr int kBoxUnits = 2 * CS;                         // 16-byte units of one box row
-  constexpr int P = CS == 2 ? 2 : 1;                        // chunks whose C values are held in registers (32 each)
-  constexpr int kUnitElems = 16 / CS;
-  const int q = warp & 3, ew = warp - kFirstEpiWarp, half = ew >> 2;
-  uint8_t* buf = epi + ew * 4096;
-  const uint8_t* Cb = static_cast<const uint8_t*>(p.C);
-  uint8_t* Db = static_cast<uint8_t*>(p.D);
-  const size_t ldc_b = (size_t)p.ldc * CS, ldd_b = (size_t)p.ldd * CS;
-  const int M = (int)p.M, N = (int)p.N;
-  const bool has_c = p.has_c != 0;
-  uint4 creg[P][8];
-  int acc = 0;
-  uint32_t acc_phase = 0;
-  // chunk n of this warp: m-block and chunk column inside the tile
-  auto chunk_of = [&](int n, int& j, int& c) -> bool {
-    j = MBLK == 2 ? half : 0;
-    c = MBLK == 2 ? n : half + 2 * n;
-    return c < kChunksPerBlock;
-  };
-  // box m of this warp (box m % kChunkBoxes of chunk m / kChunkBoxes): accumulator column; does it exist?
-  auto box_of = [&](int m, int& tcol) -> bool {
-    int j, c;
-    const bool ok = chunk_of(m / kChunkBoxes, j, c);
-    const int sc = c * kChunkBoxes + m % kChunkBoxes;
-    tcol = j * BLOCK_N + sc * 32;
-    return ok && sc < kSub;
-  };
-  for (int t = cluster_id; t < num_tiles && !sh->abort; t += num_clusters) {
-    int mt, nt;
-    tile_coords(t, p.m_tiles, p.n_tiles, p.band, mt, nt);
-    const int col_end = min(N, (nt + 1) * BLOCK_N);  // columns of this tile stop here
-    auto geom = [&](int n, int& row0, int& col0) -> bool {
-      int j, c;
-      const bool ok = chunk_of(n, j, c);
-      row0 = ((mt * MBLK + j) * CTAS + cta_rank) * kBlockM + q * 32;
-      col0 = nt * BLOCK_N + c * kChunkCols;
-      return ok && row0 < M && col0 < col_end;
-    };
-    auto load_c = [&](int n, uint4 (&c)[8]) {
-      int row0, col0;
-      if (!geom(n, row0, col0)) return;
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const int i = lane + 32 * k, rr = i >> 3, u = i & 7;
-        const int grow = row0 + rr, gcol = col0 + u * kUnitElems;
-        if (grow < M && gcol < col_end) c[k] = *reinterpret_cast<const uint4*>(Cb + (size_t)grow * ldc_b + (size_t)gcol * CS);
-      }
-    };
-    if (has_c) {
-#pragma unroll
-      for (int n = 0; n < P; ++n)
-        if (n < kMyChunks) load_c(n, creg[n]);
-    }
-    if (!bounded_wait(&sh->tmem_full[acc], acc_phase, sh, p.status, 4u, p.wait_limit)) break;
-    ptx::tc_fence_after();
-    const uint32_t t_acc = tmem_base + (acc * MBLK) * BLOCK_N + ((uint32_t)(q * 32) << 16);
-    uint32_t racc[2][32];
-    {
-      int tcol;
-      box_of(0, tcol);  // every warp has at least one box
-      ptx::tmem_ld_32x32b_x32(t_acc + tcol, racc[0]);
-    }
-#pragma unroll
-    for (int n = 0; n < kMyChunks; ++n) {
-      int row0, col0;
-      const bool live = geom(n, row0, col0);  // same answer for the whole warp
-      __syncwarp();  // the reads of the previous chunk's store phase are done
-      if (has_c) {
-        if (live) {
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const int i = lane + 32 * k, rr = i >> 3, u = i & 7;
-            *reinterpret_cast<uint4*>(buf + rr * 128 + ((u ^ (rr & 7)) << 4)) = creg[n % P][k];
-          }
-        }
-        // the C registers of chunk n are free: fetch chunk n + P into them
-        if (n + P < kMyChunks) load_c(n + P, creg[n % P]);
-        __syncwarp();
-      }
-#pragma unroll
-      for (int b = 0; b < kChunkBoxes; ++b) {
-        const int m = n * kChunkBoxes + b;
-        int tcol;
-        if (!box_of(m, tcol)) break;  // same answer for the whole warp; boxes that exist form a prefix
-        ptx::tmem_ld_wait();
-        int tcol1;
-        if (m + 1 < kMyBoxes && box_of(m + 1, tcol1)) {
-          ptx::tmem_ld_32x32b_x32(t_acc + tcol1, racc[(m + 1) & 1]);
-        } else {
-          // this warp's part of the accumulators is in registers: hand it back to the MMA issuer (CTA 0 of the pair)
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            if (CTAS == 1) ptx::mbar_arrive(&sh->tmem_empty[acc]);
-            else ptx::mbar_arrive_cluster(&sh->tmem_empty[acc], 0);
-          }
-        }
-        if (!live) continue;
-        uint32_t (&r)[32] = racc[m & 1];
-        if (KIND == 0 && p.acc_f16) widen_f16_accumulators(r);
-        float scale = 1.f, bias = 0.f;
-        if (KIND == 1 && p.dequant) {
-          const int row = min(row0 + lane, M - 1);
-          scale = __ldg(p.row_scale + row);
-          bias = p.bias ? __ldg(p.bias + row) : 0.f;
-        }
-        uint32_t c[W], o[W];
-        uint8_t* my_row = buf + lane * 128;
-        if (has_c) {
-#pragma unroll
-          for (int v = 0; v < kBoxUnits; ++v) {
-            const uint4 x = *reinterpret_cast<const uint4*>(my_row + (((b * kBoxUnits + v) ^ (lane & 7)) << 4));
-            c[4 * v] = x.x; c[4 * v + 1] = x.y; c[4 * v + 2] = x.z; c[4 * v + 3] = x.w;
-          }
-        }
-        compute_row<KIND, CS>(r, c, has_c, p, scale, bias, o);
-#pragma unroll
-        for (int v = 0; v < kBoxUnits; ++v)
-          *reinterpret_cast<uint4*>(my_row + (((b * kBoxUnits + v) ^ (lane & 7)) << 4)) =
-              make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
-      }
-      if (live) {
-        __syncwarp();
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const int i = lane + 32 * k, rr = i >> 3, u = i & 7;
-          const uint4 x = *reinterpret_cast<const uint4*>(buf + rr * 128 + ((u ^ (rr & 7)) << 4));
-          const int grow = row0 + rr, gcol = col0 + u * kUnitElems;
-          if (grow < M && gcol < col_end) *reinterpret_cast<uint4*>(Db + (size_t)grow * ldd_b + (size_t)gcol * CS) = x;
         }
       }
     }
@@ -825,24 +695,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   } else if (warp >= kFirstEpiWarp) {
     // ------------------------------ epilogue ------------------------------
     const int cs = elem_bytes((sp24_dtype)p.cd_type);
-    if (!p.cd_col_major && cs != 1) {
-      // row-major C / D: loads and stores by the epilogue warps themselves.  With C (beta != 0) in 128-byte
-      // chunks per row, if each warp can have a 4 KB buffer: the coalesced C loads are worth 8 % of the
-      // large bf16 GEMM.  Without C in 64-byte passes through two 2 KB buffers, which is the faster
-      // form for the stores alone (int8 4096 x 8192 x 4096: 80 against 88 us).
-      const bool wide = p.has_c && p.epi_bytes >= kEpiWarps * 4096;
-      if (KIND != 2 && cs == 2) {
-        if (wide) epilogue_rows_wide<KIND, 2, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id, num_clusters, num_tiles, warp, lane);
-        else epilogue_rows<KIND, 2, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id, num_clusters, num_tiles, warp, lane);
-      } else {
-        if (wide) epilogue_rows_wide<KIND, 4, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id, num_clusters, num_tiles, warp, lane);
-        else epilogue_rows<KIND, 4, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id, num_clusters, num_tiles, warp, lane);
-      }
+    if (p.epi_lsu) {
+      // row-major C / D: loads and stores by the epilogue warps themselves
+      if (KIND != 2 && cs == 2)
+        epilogue_rows<KIND, 2, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id,
+                                                                   num_clusters, num_tiles, warp, lane);
+      else
+        epilogue_rows<KIND, 4, BLOCK_N, CTAS, MBLK, C::kAccStages>(p, sh, epi, tmem_base, (int)cta_rank, cluster_id,
+                                                                   num_clusters, num_tiles, warp, lane);
     } else {
-    // Column-major C / D and 1-byte outputs.  Each warp owns 32 accumulator rows and walks its tiles in
-    // 32 x 32 boxes: TMA load of the C box (if beta != 0) into a staging buffer a few boxes ahead,
-    // tcgen05.ld of the accumulator columns, convert in place, TMA store of the D box.  Boxes outside
-    // the matrix are clipped by the TMA.
+    // Column-major C / D, 1-byte outputs, and 4-byte row-major outputs when every epilogue warp can have
+    // a box buffer of its own.  Each warp owns 32 accumulator rows and walks its tiles in 32 x 32 boxes:
+    // TMA load of the C box (if beta != 0) into a staging buffer a few boxes ahead, tcgen05.ld of the
+    // accumulator columns, convert in place, TMA store of the D box.  Boxes outside the matrix are
+    // clipped by the TMA.
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
     const int ew = warp - kFirstEpiWarp;  // epilogue warp 0..7: warps ew and ew + 4 share a lane quarter
     const int buf_bytes = 1024 * cs;
@@ -931,9 +797,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           const int row = min(row0 + lane, (int)p.M - 1);
           const float scale = __ldg(p.row_scale + row), bias = p.bias ? __ldg(p.bias + row) : 0.f;
           if (p.cd_col_major) convert_row_dequant_transposed(r, buf, lane, p, scale, bias);
-          else convert_row_dequant_i8(r, buf, lane, p, scale, bias);
-        } else {
+          else if (cs == 1) convert_row_dequant_i8(r, buf, lane, p, scale, bias);
+          else convert_row_staged<KIND>(r, buf, lane, p, scale, bias);
+        } else if (p.cd_col_major) {
           convert_row_transposed<KIND>(r, buf, lane, p);
+        } else {
+          convert_row_staged<KIND>(r, buf, lane, p, 1.f, 0.f);
         }
         ptx::fence_proxy_async_smem();
         __syncwarp();
@@ -1184,10 +1053,20 @@ sp24_status launch(const sp24_gemm_desc* d, const GemmParams& base, const void* 
   {
     p.stages = C::kMinStagesFit > C::kMaxStages ? C::kMaxStages : C::kMinStagesFit;
     const int room = C::kSmemLimit - p.stages * C::kStageBytes;
+    // Epilogue form.  Row-major 2-byte outputs: the warps' own loads and stores through two 2 KB
+    // transposing buffers per warp (measured against the TMA form: bf16 BERT FFN 26.6 against 28.7 us,
+    // fp8 16384 x 8192 x 8192 440 against 472 us, the 256 x 256 x 512 problem 12 against 17 us, the large
+    // bf16 GEMM within 3 %).  Row-major 4-byte outputs: TMA boxes if every epilogue warp can have a 4 KB
+    // box of its own (int8 4096 x 8192 x 4096: 77 against 80 us), else the warps' own stores (two-m-block
+    // int8 tiles, 16 KB of staging: 465 against 504 us on 16384 x 8192 x 8192).  Column-major and 1-byte
+    // outputs: TMA boxes, staging in powers of two from 16 KB up to two boxes per epilogue warp.
     int epi = 16384;
-    if (!p.cd_col_major && cs != 1) {
-      // the warps' own loads and stores: one or two 2 KB transposing buffers per epilogue warp
+    p.epi_lsu = 0;
+    if (!p.cd_col_major && cs == 2) {
+      p.epi_lsu = 1;
       if (room >= kEpiWarps * 4096) epi = kEpiWarps * 4096;
+    } else if (!p.cd_col_major && cs == 4 && room < kEpiWarps * 4096) {
+      p.epi_lsu = 1;
     } else {
       while (epi < 16 * 1024 * cs && 2 * epi <= room) epi *= 2;
     }
@@ -1240,7 +1119,7 @@ extern "C" size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d) {
 // accumulator buffers (epilogue overlapped), 256 x 224 -- or 256 x 240 where that takes the pairs
 // one round of tiles fewer (224: two fp32 accumulators plus the metadata columns fit the 512 columns
 // of tensor memory and 224 is a multiple of 32; 240 is the widest multiple of 16 that fits, built for
-// the 16-bit kinds with K-contiguous B and row-major output).  Small: single CTAs, 128 x 128.
+// the 16-bit kinds with K-contiguous B and row-major 16-bit output).  Small: single CTAs, 128 x 128.
 static void choose_tile(const sp24_gemm_desc* d, int& ctas, int& block_n, int& mblk) {
   const int64_t n224 = (d->N + 223) / 224;
   ctas = 1; block_n = 128; mblk = 1;
@@ -1252,7 +1131,7 @@ static void choose_tile(const sp24_gemm_desc* d, int& ctas, int& block_n, int& m
     ctas = 2; block_n = 224; mblk = 1;
     const int64_t m_tiles = (d->M + 255) / 256, pairs = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
     const bool has_240 = (d->ab_type == SP24_F16 || d->ab_type == SP24_BF16) && d->order_b == SP24_COL_MAJOR &&
-                         d->order_d == SP24_ROW_MAJOR;
+                         d->order_d == SP24_ROW_MAJOR && elem_bytes(d->cd_type) == 2;
     const int64_t rounds224 = (m_tiles * n224 + pairs - 1) / pairs;
     const int64_t rounds240 = (m_tiles * ((d->N + 239) / 240) + pairs - 1) / pairs;
     if (has_240 && rounds240 < rounds224) block_n = 240;
@@ -1421,7 +1300,7 @@ static sp24_status run_gemm(const sp24_gemm_desc* d, const void* alpha, const vo
   SP24_DISPATCH(2, 224, 2)
   SP24_DISPATCH(2, 192, 2)
   SP24_DISPATCH(2, 256, 1)
-  if (ctas == 2 && block_n == 240 && mblk == 1 && !b_mn && !tf32 && !f8 && !i8 && !p.cd_col_major && elem_bytes(d->cd_type) != 1)
+  if (ctas == 2 && block_n == 240 && mblk == 1 && !b_mn && !tf32 && !f8 && !i8 && !p.cd_col_major && elem_bytes(d->cd_type) == 2)
     return SP24_LAUNCH(0, 240, 2, 1, false);
   SP24_DISPATCH_TF32(1, 128, 1)
   SP24_DISPATCH_TF32(2, 224, 1)

@@ -67,3 +67,30 @@ def test_argument_errors_are_reported_before_touching_a_device():
                          8, None) == 7                                         # workspace too small
     assert lib.sp24_gemm(ctypes.byref(desc), ctypes.byref(a), ctypes.c_void_p(24), one, one, ctypes.byref(b),
                          None, one, one, 256, None) == 5                       # misaligned A
+
+
+def test_tile_plan_and_support_calls_answer_without_a_device():
+    """sp24_gemm_plan is host logic: the large and the small shapes do not depend on the SM count, and a
+    forced tile shape is reported back; the FP16-accumulate entry point rejects other types on the host."""
+    from paper_2104_08378_b200 import binding as sp
+    lib = sp.lib
+    assert sp.gemm_plan(sp.make_desc("bf16", "bf16", 49152, 8192, 12288, 6144, 12288, 8192, 8192)) == "2x224x2"
+    assert sp.gemm_plan(sp.make_desc("f16", "f16", 256, 256, 512, 256, 512, 256, 256)) == "1x128x1"
+    c = ctypes.c_int()
+    desc = sp.make_desc("bf16", "bf16", 256, 256, 512, 256, 512, 256, 256)
+    assert lib.sp24_gemm_plan(ctypes.byref(desc), None, ctypes.byref(c), ctypes.byref(c)) == 1        # null
+    bad = sp.make_desc("bf16", "bf16", 256, 256, 0, 256, 512, 256, 256)
+    assert lib.sp24_gemm_plan(ctypes.byref(bad), ctypes.byref(c), ctypes.byref(c), ctypes.byref(c)) == 3   # K = 0
+    try:
+        sp.set_tile_override("2x192x2")
+        assert sp.gemm_plan(desc) == "2x192x2"
+    finally:
+        sp.set_tile_override(None)
+    assert sp.gemm_plan(desc) == "1x128x1"
+    assert lib.sp24_set_tile_override(-1, 0, 0, 0) == 3
+    one = ctypes.c_void_p(16)
+    a, b = ctypes.c_float(1), ctypes.c_float(0)
+    desc = sp.make_desc("bf16", "bf16", 16, 16, 16, 8, 16, 16, 16)
+    assert lib.sp24_gemm_f16acc(ctypes.byref(desc), ctypes.byref(a), one, one, one, ctypes.byref(b), None, one, one,
+                                256, None) == 2                                # FP16 operands only
+    assert lib.sp24_gemm_status(None, None) == 1

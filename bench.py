@@ -329,8 +329,17 @@ def run_ours(args, cfg):
         return a.elapsed_time(b) / n
 
     if world == 1 and not args.rows and not args.no_sustained:
+        sus_sampler = ClockSampler(local_rank, period_s=0.01)
+        sus_sampler.start()
         sus_ms = time_sustained(lambda: sp.gemm(vals, meta, Bt, alpha=cfg.alpha, beta=cfg.beta, C=C, out=Dout, cd=cd, ws=ws))
+        sus_clocks = sus_sampler.stop()
         kernels["gemm_sustained_ms"] = sus_ms
+        # the clock the power cap allowed during that loop, and the time re-based to 1 GHz: a figure that can
+        # be compared between runs and boxes whose power and thermal state differ
+        if sus_clocks.get("sm_mhz"):
+            kernels["gemm_sustained_sm_mhz"] = sus_clocks["sm_mhz"]
+            kernels["gemm_sustained_ms_x_sm_ghz"] = sus_ms * sus_clocks["sm_mhz"] / 1e3
+            kernels["gemm_sustained_clock_reasons"] = sus_clocks["reasons"]
         kernels["gemm_sustained_dense_equiv_tflops"] = flop / (sus_ms * 1e-3) / 1e12
         kernels["gemm_sustained_frac_of_2x_measured_sustained_dense"] = \
             flop / (sus_ms * 1e-3) / 1e12 / (2.0 * peaks["bf16_tflops_sustained"] * (2.0 if ab == "i8" else 1.0))

@@ -15,9 +15,11 @@ from test_gpu_gemm import check_fp
 pytestmark = pytest.mark.gpu
 
 TORCH_F8 = {"e4m3": torch.float8_e4m3fn, "e5m2": torch.float8_e5m2}
-TILES = ["1x128x1", "2x224x1", "2x224x2", "2x192x2", "2x256x1", "2x240x1"]
+TILES = ["1x128x1", "2x224x1", "2x224x2", "2x192x2", "2x256x1", "2x240x1", "2x256x2"]
+DENSE_ONLY = {"2x256x2"}          # two 256-column accumulators fill tensor memory: no room for metadata columns
 NO_192 = [t for t in TILES if t not in ("2x192x2", "2x240x1")]
-BUILT = {"bf16": TILES, "f16": TILES, "i8": TILES[:5], "tf32": NO_192, "e4m3": NO_192, "e5m2": NO_192}
+BUILT = {"bf16": TILES, "f16": TILES, "i8": [t for t in TILES if t != "2x240x1"], "tf32": NO_192[:4], "e4m3": NO_192,
+         "e5m2": NO_192}
 
 
 @pytest.fixture(scope="module")
@@ -38,7 +40,7 @@ def _dev(a, kind):
 @pytest.mark.parametrize("tile", TILES)
 @pytest.mark.parametrize("kind", ["bf16", "f16", "i8", "tf32", "e4m3", "e5m2"])
 def test_forced_tile_shape(sp, force_tile, kind, tile, dense):
-    if tile not in BUILT[kind]:
+    if tile not in BUILT[kind] or (tile in DENSE_ONLY and not dense):
         pytest.skip("shape not built for this kind")
     M, N, K = 1184, 736, 640          # 2.3 tiles of 512 rows, 3.3 of 224 columns, 5 k-blocks of 128
     A = inputs._matrix(("int8",) if kind == "i8" else ("normal", 1.0), kind, 21, 5, K, 0, M)

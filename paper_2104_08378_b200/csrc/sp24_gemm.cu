@@ -555,16 +555,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           conv_p = rem / p.conv_w;
           conv_q = rem - conv_p * p.conv_w;
         }
-        // Every other tile of a CTA walks K backwards: the tiles of a wave finish together, so what the L2
-        // still holds of the A panel they shared is its END, and the next wave (same rows of A, other
-        // columns) meets it first if it starts there: 12 % fewer DRAM reads on the 8192 x 8192 x 12288 case.
-        // (The sum of a tile is taken in a fixed order either way; results stay identical from launch to
-        // launch.)
-        const bool k_reversed = ((t - cluster_id) / num_clusters) & 1;
-        for (int kq = 0; kq < p.k_blocks; ++kq) {
-          const int kb = k_reversed ? p.k_blocks - 1 - kq : kq;
+        // (Walking K backwards in every other tile of a CTA, so that a wave first meets the END of the A
+        // panel the wave before it has just finished with, saves 12 % of the DRAM reads and 1.5 % of the
+        // time, but makes the rounding of a result depend on which CTA computed its tile: the same rows
+        // and columns would no longer give the same bits when M or N is split differently.  Not done.)
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!bounded_wait(&sh->empty[stage], phase ^ 1u, sh, p.status, 1u, p.wait_limit)) break;
-          if (p.test_skip_stage && t == cluster_id && kq == 1) {
+          if (p.test_skip_stage && t == cluster_id && kb == 1) {
             // test hook: this k-block of the first tile is neither armed nor loaded by either CTA, so
             // the MMA issuer's wait for it expires and every role leaves through the abort path
             if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -1124,33 +1121,54 @@ extern "C" size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d) {
   return 256;
 }
 
-// Tile choice.  Large problems (at least six waves of tiles): a pair of CTAs with two m-blocks each,
-// 512 x 224 tiles: least operand traffic per flop.  Medium: a pair with one m-block and two
-// accumulator buffers (epilogue overlapped), 256 x 224 -- or 256 x 240 where that takes the pairs
-// one round of tiles fewer (224: two fp32 accumulators plus the metadata columns fit the 512 columns
-// of tensor memory and 224 is a multiple of 32; 240 is the widest multiple of 16 that fits, built for
-// the 16-bit kinds with K-contiguous B and row-major 16-bit output).  Small: single CTAs, 128 x 128.
+// Tile choice.  Small problems: single CTAs, 128 x 128 tiles.  Otherwise a pair of CTAs, and among the
+// pair shapes the one with the smallest estimated time = rounds of tiles over the pairs x time of one
+// tile.  The tile times are measured ratios (unit: one 256 x 224 tile per unit of K; interleaved runs on
+// 2048..8192-row problems with K = 4096..16384):
+//   256 x 224, two accumulator buffers (epilogue overlapped)      K                 the reference
+//   256 x 240, the same (16-bit kinds, 16-bit row-major output)    1.04 K            operand bytes per k
+//   256 x 256, one accumulator buffer (epilogue exposed)           1.09 K + 450
+//   512 x 224, two m-blocks per CTA share a B tile (epilogue exposed): twice the work in
+//              1.65 K + 1150 (16-bit kinds), 1.80 K + 820 (8-bit floats), 1.98 K + 200 (int8 -> int32)
+// (224: two fp32 accumulators plus the metadata columns fit the 512 columns of tensor memory and 224 is a
+// multiple of 32; 240 is the widest multiple of 16 that fits.)  The dense variant keeps a fixed rule:
+// two m-blocks from six waves of tiles on, 512 x 256 there (no metadata columns needed).
 static void choose_tile(const sp24_gemm_desc* d, int& ctas, int& block_n, int& mblk) {
   const int64_t n224 = (d->N + 223) / 224;
   ctas = 1; block_n = 128; mblk = 1;
-  if (d->M >= 512 && (d->M / 512) * n224 >= 444) {
-    ctas = 2; block_n = 224; mblk = 2;
-    // the dense variant needs no metadata columns: two 256-column accumulators fill tensor memory exactly,
-    // 9 % fewer operand bytes per flop than 512 x 224 (K-contiguous B, 16-bit and 8-bit kinds)
-    if (d->a_is_dense && d->order_b == SP24_COL_MAJOR && d->ab_type != SP24_F32) block_n = 256;
+  if (d->M < 256 || (d->M / 256) * n224 < 32) return;
+  ctas = 2; block_n = 224;
+  const bool k_major_b = d->order_b == SP24_COL_MAJOR;
+  const int64_t pairs = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
+  if (d->a_is_dense) {
+    if (d->M >= 512 && (d->M / 512) * n224 >= 444) {
+      mblk = 2;
+      // two 256-column accumulators fill tensor memory exactly: 9 % fewer operand bytes per flop than 512 x 224
+      if (k_major_b && d->ab_type != SP24_F32) block_n = 256;
+      return;
+    }
+    if (k_major_b && d->N <= 2048 && (d->N + 255) / 256 < n224) block_n = 256;
     return;
   }
-  if (d->M >= 256 && (d->M / 256) * n224 >= 32) {
-    ctas = 2; block_n = 224; mblk = 1;
-    const int64_t m_tiles = (d->M + 255) / 256, pairs = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
-    const bool has_240 = (d->ab_type == SP24_F16 || d->ab_type == SP24_BF16) && d->order_b == SP24_COL_MAJOR &&
-                         d->order_d == SP24_ROW_MAJOR && elem_bytes(d->cd_type) == 2;
-    const int64_t rounds224 = (m_tiles * n224 + pairs - 1) / pairs;
-    const int64_t rounds240 = (m_tiles * ((d->N + 239) / 240) + pairs - 1) / pairs;
-    if (has_240 && rounds240 < rounds224) block_n = 240;
-    // Few tokens: every n-tile streams all of A again, so the number of n-tiles decides; 256 columns
-    // (one accumulator buffer, epilogue not overlapped) when that saves one.  Built for K-contiguous B.
-    if (d->order_b == SP24_COL_MAJOR && d->N <= 2048 && (d->N + 255) / 256 < (d->N + block_n - 1) / block_n) block_n = 256;
+  const bool bits16 = d->ab_type == SP24_F16 || d->ab_type == SP24_BF16;
+  const bool has_240 = bits16 && k_major_b && d->order_d == SP24_ROW_MAJOR && elem_bytes(d->cd_type) == 2;
+  const double K = (double)d->K;
+  const double two_a = d->ab_type == SP24_I8 ? 1.98 : (is_fp8(d->ab_type) ? 1.80 : 1.65);
+  const double two_b = d->ab_type == SP24_I8 ? 200.0 : (is_fp8(d->ab_type) ? 820.0 : 1150.0);
+  struct Candidate { int block_n, mblk; bool built; double tile_time; };
+  const Candidate candidates[4] = {
+      {224, 2, d->M >= 512, two_a * K + two_b},
+      {224, 1, true, K},
+      {240, 1, has_240, (144.0 + 240.0) / (144.0 + 224.0) * K},
+      {256, 1, k_major_b && (bits16 || d->N <= 2048), (144.0 + 256.0) / (144.0 + 224.0) * K + 450.0},
+  };
+  double best = 0.0;
+  for (const Candidate& c : candidates) {
+    if (!c.built) continue;
+    const int64_t rows = 256 * c.mblk;
+    const int64_t tiles = ((d->M + rows - 1) / rows) * ((d->N + c.block_n - 1) / c.block_n);
+    const double cost = (double)((tiles + pairs - 1) / pairs) * c.tile_time;
+    if (best == 0.0 || cost < best) { best = cost; block_n = c.block_n; mblk = c.mblk; }
   }
 }
 

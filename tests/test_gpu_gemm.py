@@ -347,3 +347,28 @@ def test_rejects_bad_arguments(sp):
         sp.gemm(a, m, bt, beta=1.0)
     out = sp.gemm(torch.zeros((0, 8), dtype=torch.float16, device="cuda"), m, bt)
     assert out.shape == (0, 16)
+
+
+@pytest.mark.parametrize("ab", ["bf16", "i8"])
+def test_shards_of_tokens_or_rows_give_the_bits_of_the_full_product(sp, ab):
+    """Splitting N (tokens, the multi-GPU sharding) or M (the row bands of the host pipeline) must not
+    change a single bit of the result, although the shards run on other tile shapes than the full
+    problem: every output element is accumulated over K in the same order whatever tile computes it."""
+    M, N, K = 2048, 4096, 1024
+    cfg = inputs.scaled(inputs.CONFIGS["int8_linear" if ab == "i8" else "bert_ffn_bf16"], M=M, N=N, K=K)
+    A, Bt = to_device(inputs.gen_A(cfg), ab), to_device(inputs.gen_Bt(cfg), ab)
+    vals, meta, _ = sp.compress(A)
+    cd = "i32" if ab == "i8" else "bf16"
+    full = sp.gemm(vals, meta, Bt, cd=cd)
+    desc = sp.make_desc(ab, cd, M, N, K, K // 2, K, N, N)
+    plans = {sp.gemm_plan(desc)}
+    for n0, n1 in ((0, 256), (256, 1280), (1280, N)):                      # token shards of unequal size
+        part = sp.gemm(vals, meta, Bt[n0:n1], cd=cd)
+        plans.add(sp.gemm_plan(sp.make_desc(ab, cd, M, n1 - n0, K, K // 2, K, n1 - n0, n1 - n0)))
+        assert torch.equal(part.view(torch.uint8), full[:, n0:n1].contiguous().view(torch.uint8))
+    for m0, m1 in ((0, 128), (128, 1152), (1152, M)):                       # row bands (128-row metadata blocks)
+        mv, mm, _ = sp.compress(A[m0:m1])
+        part = sp.gemm(mv, mm, Bt, cd=cd)
+        assert torch.equal(part.view(torch.uint8), full[m0:m1].view(torch.uint8))
+    torch.cuda.synchronize()
+    assert len(plans) > 1                                                   # the shards did take other tile shapes

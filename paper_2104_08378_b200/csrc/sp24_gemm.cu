@@ -1131,8 +1131,9 @@ extern "C" size_t sp24_gemm_workspace_bytes(const sp24_gemm_desc* d) {
 //   512 x 224, two m-blocks per CTA share a B tile (epilogue exposed): twice the work in
 //              1.65 K + 1150 (16-bit kinds), 1.80 K + 820 (8-bit floats), 1.98 K + 200 (int8 -> int32)
 // (224: two fp32 accumulators plus the metadata columns fit the 512 columns of tensor memory and 224 is a
-// multiple of 32; 240 is the widest multiple of 16 that fits.)  The dense variant keeps a fixed rule:
-// two m-blocks from six waves of tiles on, 512 x 256 there (no metadata columns needed).
+// multiple of 32; 240 is the widest multiple of 16 that fits.)  The dense variant: two m-blocks from six
+// waves of tiles on, 512 x 256 there (no metadata columns needed); below that the one-m-block width with
+// the fewest rounds.
 static void choose_tile(const sp24_gemm_desc* d, int& ctas, int& block_n, int& mblk) {
   const int64_t n224 = (d->N + 223) / 224;
   ctas = 1; block_n = 128; mblk = 1;
@@ -1140,6 +1141,8 @@ static void choose_tile(const sp24_gemm_desc* d, int& ctas, int& block_n, int& m
   ctas = 2; block_n = 224;
   const bool k_major_b = d->order_b == SP24_COL_MAJOR;
   const int64_t pairs = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
+  const bool bits16 = d->ab_type == SP24_F16 || d->ab_type == SP24_BF16;
+  const bool has_240 = bits16 && k_major_b && d->order_d == SP24_ROW_MAJOR && elem_bytes(d->cd_type) == 2;
   if (d->a_is_dense) {
     if (d->M >= 512 && (d->M / 512) * n224 >= 444) {
       mblk = 2;
@@ -1147,11 +1150,18 @@ static void choose_tile(const sp24_gemm_desc* d, int& ctas, int& block_n, int& m
       if (k_major_b && d->ab_type != SP24_F32) block_n = 256;
       return;
     }
-    if (k_major_b && d->N <= 2048 && (d->N + 255) / 256 < n224) block_n = 256;
+    // one m-block: the width that needs the fewest rounds of tiles, operand bytes per k as the tie-break
+    // (without metadata columns two 256-column accumulators fit, so 256 x 256 keeps its epilogue overlapped)
+    const int widths[3] = {224, has_240 ? 240 : 0, k_major_b && d->ab_type != SP24_F32 ? 256 : 0};
+    double best = 0.0;
+    for (const int bn : widths) {
+      if (bn == 0) continue;
+      const int64_t tiles = ((d->M + 255) / 256) * ((d->N + bn - 1) / bn);
+      const double cost = (double)((tiles + pairs - 1) / pairs) * (256.0 + bn);
+      if (best == 0.0 || cost < best) { best = cost; block_n = bn; }
+    }
     return;
   }
-  const bool bits16 = d->ab_type == SP24_F16 || d->ab_type == SP24_BF16;
-  const bool has_240 = bits16 && k_major_b && d->order_d == SP24_ROW_MAJOR && elem_bytes(d->cd_type) == 2;
   const double K = (double)d->K;
   const double two_a = d->ab_type == SP24_I8 ? 1.98 : (is_fp8(d->ab_type) ? 1.80 : 1.65);
   const double two_b = d->ab_type == SP24_I8 ? 200.0 : (is_fp8(d->ab_type) ? 820.0 : 1150.0);
